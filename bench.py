@@ -1,0 +1,398 @@
+#!/usr/bin/env python
+"""Benchmark of the failure-aware MoE routing hot path (dispatch + combine).
+
+A step is one pass of the whole path over one batch of synthetic tokens:
+gate -> mask -> top-k -> weights -> replica pick -> count/scan -> permutation
+-> scatter (dispatch), then the weighted gather-reduce (combine), on the
+DeepSeek-V3-shaped workload (T=8192, H=7168, E=256, k=8, 288 slots on 32
+simulated ranks, one rank failed).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line.  N > 1 is launched with torchrun, one rank per GPU; the
+path shards by tokens (every rank routes its own batch, no collective on the
+data path), so scaling is weak.  `--impl reference` times the CPU oracle, as it
+stands, on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "dispatch+combine tokens/s at DSv3 shape"
+UNIT = "tokens/s"
+
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from ncu captures of
+# the kernels as they stand; None when a kernel changed after its last capture.
+NCU_TRAFFIC_BYTES = {"k_scatter": None, "k_combine": None}
+
+
+def env_rank():
+    return (int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")),
+            int(os.environ.get("WORLD_SIZE", "1")))
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def algorithmic_bytes(wl, T):
+    """Bytes the method must move per launch, by kernel."""
+    row = 2 * wl.H
+    route = T * (4 * wl.E + 16 * wl.k)                 # logits in; ids, weights, slots, ranks out
+    scatter = T * ((1 + wl.k) * row + 20 * wl.k)       # x once, k copies out; slot/rank/offset in, rows out
+    combine = T * ((wl.k + 1) * row + 16 * wl.k)       # k rows in, y out; row, weight, slot, scale in
+    return {"k_route": route, "k_scatter": scatter, "k_combine": combine}
+
+
+class ClockSampler:
+    """Samples SM clock and clock-event reasons of one GPU while the timed region runs."""
+
+    def __init__(self, device_index: int, period_s: float = 0.02):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode() if hasattr(uuid, "encode") else uuid)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self._h = None
+        self.period = period_s
+
+    def _loop(self):
+        nv = self._nv
+        names = {"hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+                 "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+                 "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+                 "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4)}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self._h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
+                for n, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(n)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self._h is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        med = statistics.median(self.samples) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def oracle_cfg_for(wl):
+    import oracle
+    return oracle.OracleConfig(num_experts=wl.E, top_k=wl.k, num_ranks=wl.R, slots_per_rank=wl.S,
+                               score_func=wl.score_func, n_group=wl.n_group, topk_group=wl.topk_group)
+
+
+def oracle_step(wl, inp, failed, T):
+    """One dispatch + combine of the CPU oracle on the first T tokens."""
+    import oracle
+    from paper_2602_21140_b200 import workloads as W
+    bias = inp["bias"] if wl.score_func == W.SIGMOID else None
+    ref = oracle.dispatch(oracle_cfg_for(wl), inp["slot_to_expert"], failed, bias,
+                          inp["logits"][:T], inp["x"][:T])
+    oracle.combine(ref["send_buf"], ref["dst_row"], ref["topk_weights"], ref["topk_slot"],
+                   inp["slot_scale"])
+
+
+def time_oracle(wl, inp, failed, budget_s=12.0, t_probe=256):
+    """Oracle throughput on a bounded sample: whole steps of T_sample tokens for about budget_s."""
+    t0 = time.perf_counter()
+    oracle_step(wl, inp, failed, t_probe)
+    per_tok = (time.perf_counter() - t0) / t_probe
+    T_s = int(max(64, min(wl.T, budget_s / 3 / per_tok)))
+    n, t_start = 0, time.perf_counter()
+    while n < 3 or (time.perf_counter() - t_start < budget_s and n < 50):
+        oracle_step(wl, inp, failed, T_s)
+        n += 1
+        if time.perf_counter() - t_start > 3 * budget_s:
+            break
+    dt = time.perf_counter() - t_start
+    return {"value": T_s * n / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"{n} dispatch+combine steps over the first {T_s} of {wl.T} tokens, {dt:.1f} s, single thread"}
+
+
+def run_reference(args):
+    rank, _, world = env_rank()
+    if rank != 0:
+        return
+    from paper_2602_21140_b200 import workloads as W
+    wl = W.WORKLOADS[args.workload]
+    failed = wl.failure_sets[args.failure_set]
+    inp = W.make_inputs(wl)
+    # size the per-step sample so that warmup + steps end within about two minutes
+    t0 = time.perf_counter()
+    oracle_step(wl, inp, failed, 128)
+    per_tok = (time.perf_counter() - t0) / 128
+    T_s = int(max(8, min(wl.T, 120.0 / (args.steps + args.warmup) / per_tok)))
+    for _ in range(args.warmup):
+        oracle_step(wl, inp, failed, T_s)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(wl, inp, failed, T_s)
+    dt = time.perf_counter() - t0
+    value = T_s * args.steps / dt
+    sample = f"each step = oracle dispatch+combine over the first {T_s} of {wl.T} tokens, single thread"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": workload_name(wl, failed), "T": wl.T, "H": wl.H, "E": wl.E, "k": wl.k,
+                   "slots": wl.P, "ranks": wl.R, "failed_ranks": list(failed), "sample_tokens": T_s},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def workload_name(wl, failed):
+    return (f"{wl.name}: T={wl.T} H={wl.H} bf16, E={wl.E}, k={wl.k}, "
+            f"{'sigmoid+bias' if wl.score_func else 'softmax'}"
+            f"{f', {wl.n_group} groups top-{wl.topk_group}' if wl.n_group > 1 else ''}, "
+            f"{wl.P} slots on {wl.R} ranks, failed ranks {list(failed)}")
+
+
+def max_over_ranks(value: float, world: int, device=None) -> float:
+    """Largest `value` over all ranks (identity for a single process)."""
+    if world == 1:
+        return value
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def shard_seed(base_seed: int, rank: int) -> int:
+    """Every rank routes its own batch: same workload recipe, different seed."""
+    return base_seed + 1000 * rank
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2602_21140_b200 import binding as B
+    from paper_2602_21140_b200 import workloads as W
+
+    rank, local_rank, world = env_rank()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    wl = W.WORKLOADS[args.workload]
+    failed = wl.failure_sets[args.failure_set]
+    T, K, Wm = wl.T, args.steps, args.warmup
+    inp = W.make_inputs(wl, seed=shard_seed(wl.seed, rank))
+    bias = inp["bias"] if wl.score_func == W.SIGMOID else None
+    router = B.MoeRouter(B.config_for_workload(wl), inp["slot_to_expert"], bias, inp["slot_scale"], device=dev)
+    router.set_failed_ranks(failed)
+
+    lg_h = torch.from_numpy(inp["logits"]).pin_memory()
+    x_h = torch.from_numpy(inp["x"]).view(torch.int16).view(torch.bfloat16).pin_memory()
+    y_h = torch.empty((T, wl.H), dtype=torch.bfloat16).pin_memory()
+    logits, x = lg_h.to(dev), x_h.to(dev)
+    out = router.alloc_outputs(T)
+    y = torch.empty((T, wl.H), dtype=torch.bfloat16, device=dev)
+
+    stream = torch.cuda.Stream(device=dev)
+    stream.wait_stream(torch.cuda.current_stream())
+    launches = 0
+    with torch.cuda.stream(stream):
+        for _ in range(max(Wm, 3)):
+            router.dispatch(logits, x, out)
+            router.combine(out.send_buf, T, y)
+        stream.synchronize()
+        assert router.device_status() == 0
+        assert int(out.slot_offsets[-1]) == T * wl.k
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            router.dispatch(logits, x, out)
+            router.combine(out.send_buf, T, y)
+        for _ in range(max(Wm, 3)):
+            graph.replay()
+        stream.synchronize()
+
+        # ---- timed region: K replays of the captured step -----------------
+        sampler = ClockSampler(local_rank)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sampler.start()
+        e0.record(stream)
+        for _ in range(K):
+            graph.replay()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        clocks = sampler.stop()
+        if world > 1:
+            dist.barrier()
+        ms_total = max_over_ranks(e0.elapsed_time(e1), world, dev)
+        launches += 3 * K
+        value = world * T * K / (ms_total * 1e-3)
+
+        # ---- per-kernel durations: eager launches with events between the kernels
+        K2 = min(K, 200)
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K2)]
+        for i in range(K2):
+            router.set_timing_event(ev[i][1])
+            ev[i][0].record(stream)
+            router.dispatch(logits, x, out)
+            ev[i][2].record(stream)
+            router.combine(out.send_buf, T, y)
+            ev[i][3].record(stream)
+        router.set_timing_event(None)
+        torch.cuda.synchronize()
+        launches += 3 * K2
+        dur_ms = {"k_route": statistics.mean(e[0].elapsed_time(e[1]) for e in ev),
+                  "k_scatter": statistics.mean(e[1].elapsed_time(e[2]) for e in ev),
+                  "k_combine": statistics.mean(e[2].elapsed_time(e[3]) for e in ev)}
+
+        # ---- end to end through the C ABI with host buffers ----------------
+        K3 = min(K, 20)
+        lg_d, x_d = torch.empty_like(logits), torch.empty_like(x)
+        for _ in range(2):
+            router.step_host(lg_h, x_h, out, lg_d, x_d, y, y_h)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(K3):
+            router.step_host(lg_h, x_h, out, lg_d, x_d, y, y_h)     # returns after the D2H copy
+        e2e_s = max_over_ranks(time.perf_counter() - t0, world, dev)
+        launches += 3 * (K3 + 2)
+        e2e = {"value": world * T * K3 / e2e_s, "unit": UNIT,
+               "h2d_bytes_per_step": T * wl.E * 4 + T * wl.H * 2, "d2h_bytes_per_step": T * wl.H * 2,
+               "steps": K3, "ms_per_step": 1e3 * e2e_s / K3}
+
+        # ---- remap -> first step: same graph, no recapture ------------------
+        remap = None
+        if rank == 0:
+            import oracle
+            sets = [fs for fs in wl.failure_sets] or [()]
+            steady, with_remap, host_us = [], [], []
+            for i in range(30):
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+                graph.replay()
+                torch.cuda.synchronize()
+                steady.append(time.perf_counter() - t0)
+            for i in range(30):
+                fs = sets[i % len(sets)]
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+                router.set_failed_ranks(fs)
+                t1 = time.perf_counter()
+                graph.replay()
+                torch.cuda.synchronize()
+                with_remap.append(time.perf_counter() - t0)
+                host_us.append((t1 - t0) * 1e6)
+            launches += 60 * 3
+            # the step after the last remap is correct for the new failure set
+            ids, w, slot = oracle.route(oracle_cfg_for(wl), inp["slot_to_expert"], fs, bias, inp["logits"])
+            ok = (np.array_equal(out.topk_ids.cpu().numpy(), ids) and
+                  np.array_equal(out.topk_slot.cpu().numpy(), slot))
+            router.set_failed_ranks(failed)
+            remap = {"host_call_us_median": statistics.median(host_us),
+                     "added_latency_us_median": (statistics.median(with_remap) - statistics.median(steady)) * 1e6,
+                     "step_us_median": statistics.median(steady) * 1e6,
+                     "first_step_matches_oracle": bool(ok), "graph_recaptured": False,
+                     "failure_sets_cycled": [list(s) for s in sets]}
+        assert router.device_status() == 0
+
+    # ---- roofline of the dominant kernel -----------------------------------
+    peak, peak_kind = measured_peaks()
+    alg = algorithmic_bytes(wl, T)
+    dom = max(("k_scatter", "k_combine"), key=lambda n: dur_ms[n])
+    achieved = alg[dom] / (dur_ms[dom] * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_source": f"of {peak_kind}", "traffic": NCU_TRAFFIC_BYTES[dom],
+                "algorithmic_bytes": alg[dom], "kernel_ms": dur_ms[dom],
+                "per_kernel": {n: {"ms": dur_ms[n], "algorithmic_bytes": alg[n],
+                                   "GB/s": alg[n] / (dur_ms[n] * 1e-3) / 1e9,
+                                   "frac": alg[n] / (dur_ms[n] * 1e-3) / 1e9 / peak} for n in dur_ms},
+                "step": {"algorithmic_bytes": sum(alg.values()),
+                         "GB/s": sum(alg.values()) * K / (ms_total * 1e-3) / 1e9,
+                         "frac": sum(alg.values()) * K / (ms_total * 1e-3) / 1e9 / peak,
+                         "frac_of_8TBs_nominal": sum(alg.values()) * K / (ms_total * 1e-3) / 1e9 / 8000.0}}
+
+    cpu_baseline = None
+    if rank == 0 and world == 1:
+        cpu_baseline = time_oracle(wl, inp, failed)
+
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+            "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": workload_name(wl, failed), "T_per_gpu": T, "H": wl.H, "E": wl.E,
+                       "k": wl.k, "slots": wl.P, "ranks": wl.R, "failed_ranks": list(failed),
+                       "parallelism": f"token-sharded x{world}, no data-path collective",
+                       "l2": "working set per step 2.1 GB > 126 MB L2, no flush",
+                       "timed": "CUDA-graph replays of dispatch+combine, CUDA events, max over ranks"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
+            "cpu_baseline": cpu_baseline, "remap": remap}))
+    router.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", default="dsv3")
+    ap.add_argument("--failure-set", type=int, default=1, help="index into the workload's failure sets")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,214 @@
+/*
+ * moe_route.h — C ABI of the failure-aware MoE routing library for B200 (sm_100a).
+ *
+ * The library implements the per-layer hot path that ReviveMoE's
+ * instance-preserving recovery rewires: gate -> availability mask -> top-k ->
+ * weight renormalisation -> live-replica pick -> per-slot count and prefix
+ * scan -> stable permutation -> scatter of bf16 hidden states into an
+ * expert-contiguous send buffer (dispatch / A2E layout), and the weighted
+ * gather-reduce back to token order (combine / E2A).  Recovery is a host call
+ * that rewrites only a rank-alive bitmap and a logical-to-physical replica
+ * table held in device memory; kernels read both through pointers, so a CUDA
+ * graph captured over moe_dispatch + moe_combine stays valid after a failure.
+ *
+ * Conventions
+ *   - Every function returns a moe_status; no exception crosses this boundary.
+ *   - "host" pointers are ordinary CPU memory and are copied before return.
+ *     "device" pointers are CUDA device memory owned by the caller, on the
+ *     device that was current at moe_route_init.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *   - The context owns only small state: the routing tables, bias, per-slot
+ *     scales, scan scratch sized from max_tokens, and pinned staging buffers.
+ *   - moe_dispatch and moe_combine allocate nothing, never synchronise and
+ *     never read device memory from the host: they may be captured in a graph.
+ *   - Simulated EP ranks: slot p (0 <= p < P = num_ranks*slots_per_rank) lives
+ *     on rank p / slots_per_rank; the send buffer is one allocation in which
+ *     rank r owns rows [rank_offsets[r], rank_offsets[r+1]).
+ *   - A context is not thread-safe; serialise calls on it.
+ */
+#ifndef MOE_ROUTE_H
+#define MOE_ROUTE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct moe_ctx moe_ctx;
+
+typedef enum {
+    MOE_OK = 0,
+    MOE_ERR_INVALID_ARG = 1,          /* bad size, NULL, misaligned pointer, unsupported shape     */
+    MOE_ERR_CUDA = 2,                 /* a CUDA runtime call failed (no device, out of memory...) */
+    MOE_ERR_INSUFFICIENT_EXPERTS = 3, /* the failure set could leave a token without k experts     */
+    MOE_ERR_CAPACITY = 4,             /* T > max_tokens, or an expert has more than max_replicas   */
+    MOE_ERR_DEVICE_TIMEOUT = 5        /* a bounded device-side wait gave up (see get_device_status) */
+} moe_status;
+
+enum { MOE_SCORE_SOFTMAX = 0, MOE_SCORE_SIGMOID = 1 };
+
+/* Limits of this build: num_experts <= 512, top_k <= 16, max_replicas <= 8,
+ * num_ranks*slots_per_rank <= 4096, hidden % 8 == 0.  With n_group > 1:
+ * num_experts % n_group == 0, top_k % topk_group == 0 and top_k/topk_group
+ * in {1, 2}. */
+typedef struct {
+    int32_t num_experts;    /* E: logical experts                                            */
+    int32_t top_k;          /* k: experts per token                                          */
+    int32_t hidden;         /* H: bf16 elements per token row                                */
+    int32_t max_tokens;     /* largest T a dispatch may carry (sizes the scan scratch)       */
+    int32_t num_ranks;      /* R: simulated EP ranks                                         */
+    int32_t slots_per_rank; /* S: physical expert slots per rank                             */
+    int32_t max_replicas;   /* most physical copies any logical expert may have              */
+    int32_t score_func;     /* MOE_SCORE_SOFTMAX | MOE_SCORE_SIGMOID (+ bias on the key)     */
+    int32_t n_group;        /* 1 = plain top-k; > 1 = group-limited selection                */
+    int32_t topk_group;     /* groups kept when n_group > 1                                  */
+    int32_t replica_policy; /* 0 = replica (t mod live count) of the ascending live list     */
+    float   route_scale;    /* multiplies the renormalised weights (1.0 = weights sum to 1)  */
+} moe_config;
+
+/* Device output pointers of one dispatch.  With n = T*k:
+ *   topk_ids     [T,k] i32  chosen logical experts, best first
+ *   topk_weights [T,k] f32  renormalised gate weights
+ *   topk_slot    [T,k] i32  physical slot serving (t, j)
+ *   slot_counts  [P]   i32  assignments per slot
+ *   slot_offsets [P+1] i32  exclusive prefix of slot_counts, [P] = n
+ *   rank_counts  [R]   i32  assignments per rank (0 for a failed rank)
+ *   rank_offsets [R+1] i32  first send-buffer row of each rank, [R] = n
+ *   dst_row      [n]   i32  send-buffer row of assignment i = t*k + j
+ *   src_index    [n]   i32  inverse of dst_row
+ *   send_buf     [n,H] bf16 row dst_row[i] holds a bit copy of x[i / k]
+ * Rows of one slot keep ascending i (stable).  All pointers must be non-NULL;
+ * send_buf must be 16-byte aligned. */
+typedef struct {
+    int32_t *topk_ids;
+    float   *topk_weights;
+    int32_t *topk_slot;
+    int32_t *slot_counts;
+    int32_t *slot_offsets;
+    int32_t *rank_counts;
+    int32_t *rank_offsets;
+    int32_t *dst_row;
+    int32_t *src_index;
+    void    *send_buf;
+} moe_dispatch_out;
+
+/*
+ * moe_route_init — create a context on the current device.
+ * Sets up the routing state of Sec. 3.4: the logical-to-physical map
+ * ("which device each replica resides on") and an all-alive rank bitmap.
+ *   slot_to_expert host [P]: logical expert hosted by each physical slot, -1 = empty.
+ *   bias           host [E] or NULL: added to the selection key in sigmoid mode only.
+ *   slot_scale     host [P]: per-slot scalar standing in for the expert FFN in combine.
+ * Returns INVALID_ARG for unsupported shapes, CAPACITY if an expert exceeds
+ * max_replicas, INSUFFICIENT_EXPERTS if fewer than k experts are placed,
+ * CUDA if allocation fails.  *out is written only on success.
+ */
+moe_status moe_route_init(const moe_config *cfg, const int32_t *slot_to_expert,
+                          const float *bias, const float *slot_scale,
+                          void *cuda_stream, moe_ctx **out);
+
+/*
+ * moe_set_failed_ranks — recovery after device failures (Sec. 3.4, Sec. 4.1
+ * "update to the gating mechanism").  `ranks` host [n] is the ABSOLUTE set of
+ * failed ranks (duplicates allowed, n = 0 revives everything).  An expert
+ * whose every replica sits on a failed rank is masked before top-k ("Missing
+ * experts"); an expert with a surviving replica only stops using the failed
+ * copies ("Redundant experts").  Validates on the host; on any error the
+ * device state is untouched.  The new state is copied with one small
+ * stream-ordered transfer, so it takes effect between steps enqueued on
+ * `cuda_stream`; no graph needs recapturing.  Must not be called while the
+ * stream is capturing (INVALID_ARG).
+ */
+moe_status moe_set_failed_ranks(moe_ctx *ctx, const int32_t *ranks, int32_t n, void *cuda_stream);
+
+/*
+ * moe_update_replica_map — replace the logical-to-physical map (Sec. 3.4:
+ * removing failed replicas from the map, or placing new ones).  Same
+ * validation, ordering and capture rules as moe_set_failed_ranks; the
+ * failed-rank set is kept.
+ */
+moe_status moe_update_replica_map(moe_ctx *ctx, const int32_t *slot_to_expert, void *cuda_stream);
+
+/*
+ * moe_dispatch — gate, mask, select, count, scan, permute and scatter
+ * (Sec. 2.1 gating and top-k; Sec. 2.3 dispatch / attention2expert).
+ *   logits device [T,E] f32 row-major (finite; -inf acts as a mask)
+ *   x      device [T,H] bf16 row-major, 16-byte aligned
+ *   out    host struct of device pointers (see moe_dispatch_out)
+ * T = 0 succeeds and launches nothing.  CAPACITY if T > max_tokens.
+ */
+moe_status moe_dispatch(moe_ctx *ctx, const float *logits, const void *x, int32_t T,
+                        const moe_dispatch_out *out, void *cuda_stream);
+
+/*
+ * moe_combine — weighted gather-reduce back to token order (Sec. 2.3
+ * combine / expert2attention):
+ *   y[t,:] = bf16( sum_j (w[t,j] * slot_scale[slot[t,j]]) * expert_buf[dst_row[t*k+j], :] )
+ * with fp32 accumulation in ascending j and one rounding.  Uses the
+ * topk_weights / topk_slot / dst_row buffers of the latest moe_dispatch on
+ * this context (their pointers are remembered; the buffers stay the caller's).
+ *   expert_buf device [T*k,H] bf16 in send-buffer row order, 16-byte aligned
+ *   y          device [T,H]   bf16, 16-byte aligned
+ * INVALID_ARG if no dispatch preceded it or T differs from that dispatch.
+ */
+moe_status moe_combine(moe_ctx *ctx, const void *expert_buf, int32_t T, void *y, void *cuda_stream);
+
+/*
+ * moe_step_host — one dispatch + combine fed from HOST memory, for callers
+ * that hold activations on the CPU: copies logits and x to the given device
+ * staging buffers, runs moe_dispatch and moe_combine (expert_buf = the send
+ * buffer), copies y back and waits for the stream.  Host buffers should be
+ * pinned for the copies to be asynchronous.
+ *   logits_host [T,E] f32, x_host [T,H] bf16, y_host [T,H] bf16 (written)
+ *   logits_dev, x_dev, y_dev: device staging of the same shapes.
+ */
+moe_status moe_step_host(moe_ctx *ctx, const float *logits_host, const void *x_host, int32_t T,
+                         const moe_dispatch_out *out, float *logits_dev, void *x_dev,
+                         void *y_dev, void *y_host, void *cuda_stream);
+
+/*
+ * moe_set_timing_event — measurement hook (no counterpart in the paper).
+ * `cuda_event` is a cudaEvent_t created by the caller with timing enabled, or
+ * NULL to switch the hook off.  While set, every moe_dispatch records it on
+ * its stream between the routing kernel and the scatter kernel, so a caller
+ * bracketing moe_dispatch with its own events can split the two.  Not meant
+ * to be left on while capturing a graph.
+ */
+moe_status moe_set_timing_event(moe_ctx *ctx, void *cuda_event);
+
+/*
+ * moe_get_device_status — synchronises the device and reports whether any
+ * kernel of this context gave up on a bounded wait or met a token with fewer
+ * than k selectable experts (possible only with -inf logits).  Writes the
+ * status to *code, clears it and resets the scan scratch.  Never on the hot path.
+ */
+moe_status moe_get_device_status(moe_ctx *ctx, int32_t *code);
+
+/*
+ * moe_plan_routing_state — the host half of a remap, with no CUDA call: from a
+ * placement and a failed-rank set compute the rank-alive bitmap
+ * (ceil(R/32) words, bit r set = alive), the per-expert replica table
+ * [E, max_replicas] (ascending slot ids, -1 padded) and the number of
+ * available experts.  Any output pointer may be NULL.  Same validation and
+ * return codes as moe_set_failed_ranks.
+ */
+moe_status moe_plan_routing_state(const moe_config *cfg, const int32_t *slot_to_expert,
+                                  const int32_t *failed_ranks, int32_t n_failed,
+                                  uint32_t *rank_alive, int32_t *replica_table,
+                                  int32_t *n_available);
+
+/* Device bytes a context for `cfg` allocates (0 if cfg is invalid). */
+size_t moe_workspace_bytes(const moe_config *cfg);
+
+/* Frees the context and everything it owns.  NULL is allowed. */
+moe_status moe_route_destroy(moe_ctx *ctx);
+
+/* Static, human-readable name of a status code. */
+const char *moe_status_string(moe_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOE_ROUTE_H */

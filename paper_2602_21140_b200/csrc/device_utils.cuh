@@ -1,0 +1,124 @@
+// Device-side helpers shared by the routing, scatter and combine kernels (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace moe {
+
+// Values of the device status word (mirrors moe_status where it applies).
+constexpr int kDevOk = 0;
+constexpr int kDevInsufficientExperts = 3;   // a token met fewer than k selectable experts
+constexpr int kDevTimeout = 5;               // a bounded wait gave up
+
+// Bounded waits: polls before a waiter gives up, and the back-off between polls.
+// 1<<20 polls of >= 64 ns is well over 50 ms, far longer than any healthy step.
+constexpr unsigned kSpinLimit = 1u << 20;
+constexpr unsigned kSpinSleepNs = 64;
+
+struct Control {
+    unsigned ticket;   // next tile of the running routing kernel
+    unsigned epoch;    // step counter tagging the look-back descriptors
+    int status;        // kDev* code, sticky until the host clears it
+    int pad;
+};
+
+__device__ __forceinline__ unsigned lane_id() { return threadIdx.x & 31u; }
+
+__device__ __forceinline__ unsigned lanemask_lt()
+{
+    unsigned m;
+    asm volatile("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
+    return m;
+}
+
+__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long *p)
+{
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+
+__device__ __forceinline__ void st_relaxed_u64(unsigned long long *p, unsigned long long v)
+{
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+
+__device__ __forceinline__ unsigned ld_relaxed_u32(const unsigned *p)
+{
+    unsigned v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+__device__ __forceinline__ int ld_relaxed_s32(const int *p)
+{
+    int v;
+    asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+__device__ __forceinline__ void report_status(Control *ctl, int code)
+{
+    atomicCAS(&ctl->status, kDevOk, code);   // the first error wins and sticks
+}
+
+// 128-bit streaming accesses: the big rows are touched once per kernel, so they
+// should not displace the small routing tables from L1.
+__device__ __forceinline__ uint4 ld_stream_v4(const uint4 *p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ void st_stream_v4(uint4 *p, const uint4 &v)
+{
+    asm volatile("st.global.L1::no_allocate.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x),
+                 "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+
+// ---------------------------------------------------------------------------
+// exp / sigmoid from single IEEE fp32 operations (round to nearest even, never
+// contracted, independent of compiler flags), so that sigmoid routing keys are
+// reproducible bit for bit:
+//   n = rint(z*log2e); r = z - n*ln2 (two fused steps); degree-7 Taylor
+//   polynomial by Horner; scale by 2^n through the exponent field.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ float exp_spec(float z)
+{
+    z = fminf(fmaxf(z, -87.0f), 88.0f);
+    const float n = rintf(__fmul_rn(z, 0x1.715476p+0f));
+    float r = __fmaf_rn(-n, 0x1.62e430p-1f, z);
+    r = __fmaf_rn(-n, -0x1.05c610p-29f, r);
+    float p = 0x1.a01a02p-13f;
+    p = __fmaf_rn(p, r, 0x1.6c16c2p-10f);
+    p = __fmaf_rn(p, r, 0x1.111112p-7f);
+    p = __fmaf_rn(p, r, 0x1.555556p-5f);
+    p = __fmaf_rn(p, r, 0x1.555556p-3f);
+    p = __fmaf_rn(p, r, 0.5f);
+    p = __fmaf_rn(p, r, 1.0f);
+    p = __fmaf_rn(p, r, 1.0f);
+    const float two_n = __int_as_float((static_cast<int>(n) + 127) << 23);
+    return __fmul_rn(p, two_n);
+}
+
+__device__ __forceinline__ float sigmoid_spec(float x)
+{
+    return __fdiv_rn(1.0f, __fadd_rn(1.0f, exp_spec(-x)));
+}
+
+// Order-preserving map from fp32 to uint32 (larger float <=> larger integer),
+// with -0 folded onto +0 so that equal floats get equal codes.  0 is below the
+// code of -inf and marks "already taken / not a candidate".
+__device__ __forceinline__ uint32_t key_code(float f)
+{
+    uint32_t u = (f == 0.0f) ? 0u : __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+constexpr uint32_t kCodeNegInf = 0x007FFFFFu;   // key_code(-inf)
+
+}  // namespace moe

@@ -1,0 +1,576 @@
+// Host side of the failure-aware MoE routing library: the C ABI declared in
+// include/moe_route.h, the host half of a remap (validation, bitmap and replica
+// table), context set-up and the kernel launches.  No CPU fallback exists: every
+// step of the path runs in the kernels included below.
+#include "../../include/moe_route.h"
+
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "combine_kernels.cuh"
+#include "route_kernels.cuh"
+#include "scatter_kernels.cuh"
+
+namespace {
+
+using namespace moe;
+
+constexpr int kMaxExperts = 512;
+constexpr int kMaxTopK = 16;
+constexpr int kMaxReplicas = 8;
+constexpr int kMaxSlots = 4096;
+constexpr int kStagingSlots = 16;
+constexpr size_t kMaxSmem = 227 * 1024;
+
+// Shape-derived launch constants.
+struct Derived {
+    int E, k, H, P, R, S, max_rep;
+    int epl;               // experts per lane in the routing warp
+    int lanes_per_group;   // lanes holding one expert group (power of two), 0 if ungrouped
+    int group_m;           // keys summed into a group score
+    int rank_words;        // words of the rank bitmap
+    int state_words;       // words of the whole routing-state blob
+    int tokens_per_block;  // routing tile
+};
+
+bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
+
+bool derive(const moe_config *c, Derived *d)
+{
+    if (!c) return false;
+    if (c->num_experts < 1 || c->num_experts > kMaxExperts) return false;
+    if (c->top_k < 1 || c->top_k > kMaxTopK || c->top_k > c->num_experts) return false;
+    if (c->hidden < 8 || c->hidden % 8 != 0) return false;
+    if (c->max_tokens < 1) return false;
+    if (c->num_ranks < 1 || c->slots_per_rank < 1) return false;
+    const long long P = (long long)c->num_ranks * c->slots_per_rank;
+    if (P > kMaxSlots) return false;
+    if (c->max_replicas < 1 || c->max_replicas > kMaxReplicas) return false;
+    if (c->score_func != MOE_SCORE_SOFTMAX && c->score_func != MOE_SCORE_SIGMOID) return false;
+    if (c->replica_policy != 0) return false;
+    if (!(c->route_scale > 0.0f)) return false;
+    if ((long long)c->max_tokens * c->top_k >= (1ll << 30)) return false;   // 30-bit scan counts
+    d->E = c->num_experts; d->k = c->top_k; d->H = c->hidden; d->P = (int)P;
+    d->R = c->num_ranks; d->S = c->slots_per_rank; d->max_rep = c->max_replicas;
+    d->lanes_per_group = 0; d->group_m = 1;
+    static const int kEpl[] = {1, 2, 3, 4, 5, 6, 7, 8, 10, 12, 16};
+    d->epl = 0;
+    if (c->n_group > 1) {
+        if (c->topk_group < 1 || c->topk_group > c->n_group) return false;
+        if (d->E % c->n_group != 0 || d->k % c->topk_group != 0) return false;
+        d->group_m = d->k / c->topk_group;
+        if (d->group_m != 1 && d->group_m != 2) return false;
+        const int per = d->E / c->n_group;
+        for (int epl : kEpl) {
+            if (32 * epl < d->E || per % epl != 0) continue;
+            const int lpg = per / epl;
+            if (!is_pow2(lpg) || lpg * c->n_group > 32) continue;
+            d->epl = epl; d->lanes_per_group = lpg;
+            break;
+        }
+    } else {
+        if (c->n_group != 1) return false;
+        for (int epl : kEpl)
+            if (32 * epl >= d->E) { d->epl = epl; break; }
+    }
+    if (d->epl == 0) return false;
+    d->rank_words = (d->R + 31) / 32;
+    d->state_words = kStateHeaderWords + d->rank_words + d->E * d->max_rep;
+    d->tokens_per_block = 32;
+    if (route_smem_bytes(d->E, d->max_rep, d->tokens_per_block, d->k, d->P) > kMaxSmem - 1024)
+        return false;
+    return true;
+}
+
+// Host half of a remap (Sec. 3.4): which ranks are alive, where each expert's
+// replicas are, which experts are still served, and whether routing can always
+// find k experts.  `blob` receives the device layout documented in
+// route_kernels.cuh.
+moe_status plan_state(const moe_config *c, const Derived &d, const int32_t *slot_to_expert,
+                      const std::vector<uint8_t> &failed, std::vector<int32_t> *blob,
+                      int *n_available)
+{
+    std::vector<int32_t> out((size_t)d.state_words, -1);
+    uint32_t *alive = reinterpret_cast<uint32_t *>(out.data() + kStateHeaderWords);
+    for (int w = 0; w < d.rank_words; ++w) alive[w] = 0u;
+    for (int r = 0; r < d.R; ++r)
+        if (!failed[r]) alive[r >> 5] |= 1u << (r & 31);
+    int32_t *table = out.data() + kStateHeaderWords + d.rank_words;
+    std::vector<int> n_rep((size_t)d.E, 0), n_live((size_t)d.E, 0);
+    for (int p = 0; p < d.P; ++p) {               // ascending p keeps each row ascending
+        const int e = slot_to_expert[p];
+        if (e < 0) continue;
+        if (e >= d.E) return MOE_ERR_INVALID_ARG;
+        if (n_rep[e] == d.max_rep) return MOE_ERR_CAPACITY;
+        table[e * d.max_rep + n_rep[e]++] = p;
+        if (!failed[p / d.S]) ++n_live[e];
+    }
+    int avail = 0, fallback = -1;
+    for (int e = 0; e < d.E; ++e)
+        if (n_live[e] > 0) { ++avail; if (fallback < 0) fallback = e; }
+    bool ok;
+    if (c->n_group <= 1) {
+        ok = avail >= d.k;
+    } else {
+        // worst case: the kept groups are the non-empty ones with the fewest experts
+        const int per = d.E / c->n_group;
+        std::vector<int> cnt;
+        for (int g = 0; g < c->n_group; ++g) {
+            int a = 0;
+            for (int e = g * per; e < (g + 1) * per; ++e) a += n_live[e] > 0;
+            if (a > 0) cnt.push_back(a);
+        }
+        std::sort(cnt.begin(), cnt.end());
+        int worst = 0;
+        for (size_t i = 0; i < cnt.size() && (int)i < c->topk_group; ++i) worst += cnt[i];
+        ok = worst >= d.k;
+    }
+    if (!ok) return MOE_ERR_INSUFFICIENT_EXPERTS;
+    out[0] = fallback;
+    out[1] = avail;
+    if (blob) blob->swap(out);
+    if (n_available) *n_available = avail;
+    return MOE_OK;
+}
+
+int env_int(const char *name, int dflt)
+{
+    const char *v = std::getenv(name);
+    return (v && *v) ? std::atoi(v) : dflt;
+}
+
+}  // namespace
+
+struct moe_ctx {
+    moe_config cfg;
+    Derived d;
+    int device;
+    int sm_count;
+    // host mirror of the routing state
+    std::vector<int32_t> slot_to_expert;
+    std::vector<uint8_t> failed;
+    // device state
+    int32_t *d_state;
+    float *d_bias;
+    float *d_slot_scale;
+    unsigned long long *d_desc;
+    moe::Control *d_ctl;
+    int32_t *d_pos;
+    size_t device_bytes;
+    // pinned staging ring for stream-ordered remaps
+    int32_t *h_stage[kStagingSlots];
+    cudaEvent_t stage_done[kStagingSlots];
+    bool stage_used[kStagingSlots];
+    unsigned stage_next;
+    // launch choices
+    int scatter_impl;      // 0 = vector, 1 = bulk copies
+    int bulk_stages, bulk_ctas_per_sm;
+    int scatter_blocks_per_sm, combine_blocks_per_sm;
+    size_t route_smem;
+    // what the latest dispatch wrote, for combine
+    const float *last_weights;
+    const int32_t *last_slot;
+    const int32_t *last_dst_row;
+    int32_t last_T;
+    cudaEvent_t timing_event;   // optional: recorded between routing and scatter
+};
+
+namespace {
+
+size_t device_bytes_for(const Derived &d, int max_tokens)
+{
+    const size_t tiles = ((size_t)max_tokens + d.tokens_per_block - 1) / d.tokens_per_block;
+    size_t b = 0;
+    b += (size_t)d.state_words * 4;
+    b += (size_t)d.E * 4 + (size_t)d.P * 4;
+    b += tiles * d.P * sizeof(unsigned long long);
+    b += sizeof(moe::Control);
+    b += (size_t)max_tokens * d.k * 4;
+    return b;
+}
+
+template <int EPL>
+cudaError_t launch_route_epl(const RouteParams &p, int tiles, size_t smem, cudaStream_t st)
+{
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(k_route<EPL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    k_route<EPL><<<tiles, kRouteThreads, smem, st>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_route(int epl, const RouteParams &p, int tiles, size_t smem, cudaStream_t st)
+{
+    switch (epl) {
+        case 1: return launch_route_epl<1>(p, tiles, smem, st);
+        case 2: return launch_route_epl<2>(p, tiles, smem, st);
+        case 3: return launch_route_epl<3>(p, tiles, smem, st);
+        case 4: return launch_route_epl<4>(p, tiles, smem, st);
+        case 5: return launch_route_epl<5>(p, tiles, smem, st);
+        case 6: return launch_route_epl<6>(p, tiles, smem, st);
+        case 7: return launch_route_epl<7>(p, tiles, smem, st);
+        case 8: return launch_route_epl<8>(p, tiles, smem, st);
+        case 10: return launch_route_epl<10>(p, tiles, smem, st);
+        case 12: return launch_route_epl<12>(p, tiles, smem, st);
+        case 16: return launch_route_epl<16>(p, tiles, smem, st);
+    }
+    return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_combine(const CombineParams &p, int blocks, cudaStream_t st)
+{
+    switch (p.k) {
+        case 1: k_combine_vec<1><<<blocks, kCombineThreads, 0, st>>>(p); break;
+        case 2: k_combine_vec<2><<<blocks, kCombineThreads, 0, st>>>(p); break;
+        case 4: k_combine_vec<4><<<blocks, kCombineThreads, 0, st>>>(p); break;
+        case 6: k_combine_vec<6><<<blocks, kCombineThreads, 0, st>>>(p); break;
+        case 8: k_combine_vec<8><<<blocks, kCombineThreads, 0, st>>>(p); break;
+        default: k_combine_vec<0><<<blocks, kCombineThreads, 0, st>>>(p); break;
+    }
+    return cudaGetLastError();
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Copy `words` leading words of `blob` to the device state through a pinned
+// staging slot, ordered on `st`.  A slot is reused only after its copy has run.
+moe_status push_state(moe_ctx *ctx, const std::vector<int32_t> &blob, int words, cudaStream_t st)
+{
+    const unsigned s = ctx->stage_next % kStagingSlots;
+    if (ctx->stage_used[s] && cudaEventSynchronize(ctx->stage_done[s]) != cudaSuccess)
+        return MOE_ERR_CUDA;
+    std::memcpy(ctx->h_stage[s], blob.data(), (size_t)words * 4);
+    if (cudaMemcpyAsync(ctx->d_state, ctx->h_stage[s], (size_t)words * 4, cudaMemcpyHostToDevice,
+                        st) != cudaSuccess)
+        return MOE_ERR_CUDA;
+    if (cudaEventRecord(ctx->stage_done[s], st) != cudaSuccess) return MOE_ERR_CUDA;
+    ctx->stage_used[s] = true;
+    ctx->stage_next++;
+    return MOE_OK;
+}
+
+bool stream_is_capturing(cudaStream_t st)
+{
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cs) != cudaSuccess) { cudaGetLastError(); return false; }
+    return cs != cudaStreamCaptureStatusNone;
+}
+
+void free_ctx(moe_ctx *ctx)
+{
+    if (!ctx) return;
+    cudaFree(ctx->d_state); cudaFree(ctx->d_bias); cudaFree(ctx->d_slot_scale);
+    cudaFree(ctx->d_desc); cudaFree(ctx->d_ctl); cudaFree(ctx->d_pos);
+    for (int s = 0; s < kStagingSlots; ++s) {
+        if (ctx->h_stage[s]) cudaFreeHost(ctx->h_stage[s]);
+        if (ctx->stage_done[s]) cudaEventDestroy(ctx->stage_done[s]);
+    }
+    delete ctx;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *moe_status_string(moe_status s)
+{
+    switch (s) {
+        case MOE_OK: return "MOE_OK";
+        case MOE_ERR_INVALID_ARG: return "MOE_ERR_INVALID_ARG";
+        case MOE_ERR_CUDA: return "MOE_ERR_CUDA";
+        case MOE_ERR_INSUFFICIENT_EXPERTS: return "MOE_ERR_INSUFFICIENT_EXPERTS";
+        case MOE_ERR_CAPACITY: return "MOE_ERR_CAPACITY";
+        case MOE_ERR_DEVICE_TIMEOUT: return "MOE_ERR_DEVICE_TIMEOUT";
+    }
+    return "MOE_ERR_UNKNOWN";
+}
+
+size_t moe_workspace_bytes(const moe_config *cfg)
+{
+    Derived d;
+    if (!derive(cfg, &d)) return 0;
+    return device_bytes_for(d, cfg->max_tokens);
+}
+
+moe_status moe_plan_routing_state(const moe_config *cfg, const int32_t *slot_to_expert,
+                                  const int32_t *failed_ranks, int32_t n_failed,
+                                  uint32_t *rank_alive, int32_t *replica_table,
+                                  int32_t *n_available)
+{
+    Derived d;
+    if (!derive(cfg, &d) || !slot_to_expert || n_failed < 0 || (n_failed > 0 && !failed_ranks))
+        return MOE_ERR_INVALID_ARG;
+    std::vector<uint8_t> failed((size_t)d.R, 0);
+    for (int i = 0; i < n_failed; ++i) {
+        if (failed_ranks[i] < 0 || failed_ranks[i] >= d.R) return MOE_ERR_INVALID_ARG;
+        failed[failed_ranks[i]] = 1;
+    }
+    std::vector<int32_t> blob;
+    int avail = 0;
+    const moe_status st = plan_state(cfg, d, slot_to_expert, failed, &blob, &avail);
+    if (st != MOE_OK) return st;
+    if (rank_alive) std::memcpy(rank_alive, blob.data() + kStateHeaderWords, (size_t)d.rank_words * 4);
+    if (replica_table)
+        std::memcpy(replica_table, blob.data() + kStateHeaderWords + d.rank_words,
+                    (size_t)d.E * d.max_rep * 4);
+    if (n_available) *n_available = avail;
+    return MOE_OK;
+}
+
+moe_status moe_route_init(const moe_config *cfg, const int32_t *slot_to_expert, const float *bias,
+                          const float *slot_scale, void *cuda_stream, moe_ctx **out)
+{
+    Derived d;
+    if (!out || !slot_to_expert || !slot_scale || !derive(cfg, &d)) return MOE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    std::vector<uint8_t> failed((size_t)d.R, 0);
+    std::vector<int32_t> blob;
+    moe_status ms = plan_state(cfg, d, slot_to_expert, failed, &blob, nullptr);
+    if (ms != MOE_OK) return ms;
+
+    moe_ctx *ctx = new (std::nothrow) moe_ctx();
+    if (!ctx) return MOE_ERR_CUDA;
+    ctx->cfg = *cfg; ctx->d = d;
+    ctx->slot_to_expert.assign(slot_to_expert, slot_to_expert + d.P);
+    ctx->failed = failed;
+    ctx->last_weights = nullptr; ctx->last_slot = nullptr; ctx->last_dst_row = nullptr;
+    ctx->last_T = -1;
+    ctx->timing_event = nullptr;
+    ctx->stage_next = 0;
+    for (int s = 0; s < kStagingSlots; ++s) {
+        ctx->h_stage[s] = nullptr; ctx->stage_done[s] = nullptr; ctx->stage_used[s] = false;
+    }
+    ctx->d_state = nullptr; ctx->d_bias = nullptr; ctx->d_slot_scale = nullptr;
+    ctx->d_desc = nullptr; ctx->d_ctl = nullptr; ctx->d_pos = nullptr;
+
+    bool ok = cudaGetDevice(&ctx->device) == cudaSuccess &&
+              cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device) ==
+                  cudaSuccess;
+    const size_t tiles = ((size_t)cfg->max_tokens + d.tokens_per_block - 1) / d.tokens_per_block;
+    ok = ok && cudaMalloc(&ctx->d_state, (size_t)d.state_words * 4) == cudaSuccess;
+    ok = ok && cudaMalloc(&ctx->d_bias, (size_t)d.E * 4) == cudaSuccess;
+    ok = ok && cudaMalloc(&ctx->d_slot_scale, (size_t)d.P * 4) == cudaSuccess;
+    ok = ok && cudaMalloc(&ctx->d_desc, tiles * d.P * sizeof(unsigned long long)) == cudaSuccess;
+    ok = ok && cudaMalloc(&ctx->d_ctl, sizeof(moe::Control)) == cudaSuccess;
+    ok = ok && cudaMalloc(&ctx->d_pos, (size_t)cfg->max_tokens * d.k * 4) == cudaSuccess;
+    for (int s = 0; s < kStagingSlots && ok; ++s) {
+        ok = cudaMallocHost(&ctx->h_stage[s], (size_t)d.state_words * 4) == cudaSuccess &&
+             cudaEventCreateWithFlags(&ctx->stage_done[s], cudaEventDisableTiming) == cudaSuccess;
+    }
+    ctx->device_bytes = device_bytes_for(d, cfg->max_tokens);
+    if (ok) {
+        std::vector<float> b((size_t)d.E, 0.0f);
+        if (bias) std::copy(bias, bias + d.E, b.begin());
+        const moe::Control c0 = {0u, 1u, kDevOk, 0};
+        // synchronous pageable copies: the host arrays may be freed on return
+        ok = cudaMemsetAsync(ctx->d_desc, 0, tiles * d.P * sizeof(unsigned long long), st) == cudaSuccess &&
+             cudaMemcpyAsync(ctx->d_ctl, &c0, sizeof(c0), cudaMemcpyHostToDevice, st) == cudaSuccess &&
+             cudaMemcpyAsync(ctx->d_bias, b.data(), (size_t)d.E * 4, cudaMemcpyHostToDevice, st) == cudaSuccess &&
+             cudaMemcpyAsync(ctx->d_slot_scale, slot_scale, (size_t)d.P * 4, cudaMemcpyHostToDevice, st) == cudaSuccess &&
+             cudaMemcpyAsync(ctx->d_state, blob.data(), (size_t)d.state_words * 4, cudaMemcpyHostToDevice, st) == cudaSuccess &&
+             cudaStreamSynchronize(st) == cudaSuccess;
+    }
+    if (ok) {
+        ctx->route_smem = route_smem_bytes(d.E, d.max_rep, d.tokens_per_block, d.k, d.P);
+        ctx->scatter_impl = env_int("MOE_SCATTER_IMPL", 0);
+        ctx->bulk_stages = std::min(8, std::max(1, env_int("MOE_BULK_STAGES", 4)));
+        const size_t stage_bytes = ((size_t)d.H * 2 + 127) & ~(size_t)127;
+        while (ctx->bulk_stages > 1 && ctx->bulk_stages * stage_bytes > kMaxSmem - 2048) --ctx->bulk_stages;
+        if (ctx->bulk_stages * stage_bytes > kMaxSmem - 2048) ctx->scatter_impl = 0;   // row too wide to stage
+        const size_t ring = ctx->bulk_stages * stage_bytes;
+        int fit = (int)((kMaxSmem - 1024) / (ring + 1024));
+        ctx->bulk_ctas_per_sm = std::min(32, std::max(1, env_int("MOE_BULK_CTAS_PER_SM", fit)));
+        if (ctx->bulk_ctas_per_sm > fit) ctx->bulk_ctas_per_sm = std::max(1, fit);
+        if (ctx->scatter_impl == 1)
+            ok = cudaFuncSetAttribute(k_scatter_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)ring) == cudaSuccess;
+        ctx->scatter_blocks_per_sm = std::max(1, env_int("MOE_SCATTER_BLOCKS_PER_SM", 8));
+        ctx->combine_blocks_per_sm = std::max(1, env_int("MOE_COMBINE_BLOCKS_PER_SM", 8));
+    }
+    if (!ok) {
+        cudaGetLastError();
+        free_ctx(ctx);
+        return MOE_ERR_CUDA;
+    }
+    *out = ctx;
+    return MOE_OK;
+}
+
+moe_status moe_set_failed_ranks(moe_ctx *ctx, const int32_t *ranks, int32_t n, void *cuda_stream)
+{
+    if (!ctx || n < 0 || (n > 0 && !ranks)) return MOE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const Derived &d = ctx->d;
+    std::vector<uint8_t> failed((size_t)d.R, 0);
+    for (int i = 0; i < n; ++i) {
+        if (ranks[i] < 0 || ranks[i] >= d.R) return MOE_ERR_INVALID_ARG;
+        failed[ranks[i]] = 1;
+    }
+    std::vector<int32_t> blob;
+    const moe_status ms = plan_state(&ctx->cfg, d, ctx->slot_to_expert.data(), failed, &blob, nullptr);
+    if (ms != MOE_OK) return ms;
+    if (stream_is_capturing(st)) return MOE_ERR_INVALID_ARG;
+    // only the header and the rank bitmap change
+    const moe_status ps = push_state(ctx, blob, kStateHeaderWords + d.rank_words, st);
+    if (ps == MOE_OK) ctx->failed.swap(failed);
+    return ps;
+}
+
+moe_status moe_update_replica_map(moe_ctx *ctx, const int32_t *slot_to_expert, void *cuda_stream)
+{
+    if (!ctx || !slot_to_expert) return MOE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const Derived &d = ctx->d;
+    std::vector<int32_t> blob;
+    const moe_status ms = plan_state(&ctx->cfg, d, slot_to_expert, ctx->failed, &blob, nullptr);
+    if (ms != MOE_OK) return ms;
+    if (stream_is_capturing(st)) return MOE_ERR_INVALID_ARG;
+    const moe_status ps = push_state(ctx, blob, d.state_words, st);
+    if (ps == MOE_OK) ctx->slot_to_expert.assign(slot_to_expert, slot_to_expert + d.P);
+    return ps;
+}
+
+moe_status moe_dispatch(moe_ctx *ctx, const float *logits, const void *x, int32_t T,
+                        const moe_dispatch_out *out, void *cuda_stream)
+{
+    if (!ctx || !out || T < 0) return MOE_ERR_INVALID_ARG;
+    if (T > ctx->cfg.max_tokens) return MOE_ERR_CAPACITY;
+    if (T == 0) {                     // nothing to route: no launch, pointers not inspected
+        ctx->last_weights = out->topk_weights; ctx->last_slot = out->topk_slot;
+        ctx->last_dst_row = out->dst_row; ctx->last_T = 0;
+        return MOE_OK;
+    }
+    if (!out->topk_ids || !out->topk_weights || !out->topk_slot || !out->slot_counts ||
+        !out->slot_offsets || !out->rank_counts || !out->rank_offsets || !out->dst_row ||
+        !out->src_index || !out->send_buf)
+        return MOE_ERR_INVALID_ARG;
+    if (!logits || !x) return MOE_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(out->send_buf) || !aligned16(logits)) return MOE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const Derived &d = ctx->d;
+    ctx->last_weights = out->topk_weights; ctx->last_slot = out->topk_slot;
+    ctx->last_dst_row = out->dst_row; ctx->last_T = T;
+
+    RouteParams rp;
+    rp.logits = logits; rp.T = T; rp.E = d.E; rp.k = d.k; rp.P = d.P; rp.R = d.R; rp.S = d.S;
+    rp.max_rep = d.max_rep; rp.score_func = ctx->cfg.score_func; rp.n_group = ctx->cfg.n_group;
+    rp.topk_group = ctx->cfg.topk_group; rp.lanes_per_group = d.lanes_per_group;
+    rp.group_m = d.group_m; rp.route_scale = ctx->cfg.route_scale;
+    rp.tokens_per_block = d.tokens_per_block; rp.rank_words = d.rank_words;
+    rp.state = ctx->d_state; rp.bias = ctx->d_bias;
+    rp.topk_ids = out->topk_ids; rp.topk_weights = out->topk_weights; rp.topk_slot = out->topk_slot;
+    rp.pos_in_slot = ctx->d_pos;
+    rp.slot_counts = out->slot_counts; rp.slot_offsets = out->slot_offsets;
+    rp.rank_counts = out->rank_counts; rp.rank_offsets = out->rank_offsets;
+    rp.desc = ctx->d_desc; rp.ctl = ctx->d_ctl;
+    const int tiles = (T + d.tokens_per_block - 1) / d.tokens_per_block;
+    if (launch_route(d.epl, rp, tiles, ctx->route_smem, st) != cudaSuccess) return MOE_ERR_CUDA;
+    if (ctx->timing_event && cudaEventRecord(ctx->timing_event, st) != cudaSuccess) return MOE_ERR_CUDA;
+
+    ScatterParams sp;
+    sp.x = static_cast<const uint4 *>(x); sp.send = static_cast<uint4 *>(out->send_buf);
+    sp.T = T; sp.k = d.k; sp.hv = d.H / 8;
+    sp.topk_slot = out->topk_slot; sp.slot_offsets = out->slot_offsets; sp.pos_in_slot = ctx->d_pos;
+    sp.dst_row = out->dst_row; sp.src_index = out->src_index; sp.ctl = ctx->d_ctl;
+    if (ctx->scatter_impl == 1) {
+        const unsigned stage_bytes = ((unsigned)d.H * 2u + 127u) & ~127u;
+        const int grid = std::min(T, ctx->sm_count * ctx->bulk_ctas_per_sm);
+        k_scatter_bulk<<<grid, kBulkThreads, (size_t)ctx->bulk_stages * stage_bytes, st>>>(sp, ctx->bulk_stages);
+    } else {
+        const int chunks = (sp.hv + kScatterChunk - 1) / kScatterChunk;
+        const long long items = (long long)T * chunks;
+        const long long want = (items + kScatterThreads / 32 - 1) / (kScatterThreads / 32);
+        const int grid = (int)std::min<long long>(want, (long long)ctx->sm_count * ctx->scatter_blocks_per_sm);
+        k_scatter_vec<<<grid, kScatterThreads, 0, st>>>(sp);
+    }
+    if (cudaGetLastError() != cudaSuccess) return MOE_ERR_CUDA;
+    return MOE_OK;
+}
+
+moe_status moe_combine(moe_ctx *ctx, const void *expert_buf, int32_t T, void *y, void *cuda_stream)
+{
+    if (!ctx || T < 0) return MOE_ERR_INVALID_ARG;
+    if (ctx->last_T < 0 || T != ctx->last_T) return MOE_ERR_INVALID_ARG;
+    if (T == 0) return MOE_OK;
+    if (!expert_buf || !y || !aligned16(expert_buf) || !aligned16(y)) return MOE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const Derived &d = ctx->d;
+    CombineParams cp;
+    cp.buf = static_cast<const uint4 *>(expert_buf); cp.y = static_cast<uint4 *>(y);
+    cp.T = T; cp.k = d.k; cp.hv = d.H / 8;
+    cp.dst_row = ctx->last_dst_row; cp.topk_weights = ctx->last_weights; cp.topk_slot = ctx->last_slot;
+    cp.slot_scale = ctx->d_slot_scale;
+    const int chunks = (cp.hv + kCombineChunk - 1) / kCombineChunk;
+    const long long items = (long long)T * chunks;
+    const long long want = (items + kCombineThreads / 32 - 1) / (kCombineThreads / 32);
+    const int grid = (int)std::min<long long>(want, (long long)ctx->sm_count * ctx->combine_blocks_per_sm);
+    if (launch_combine(cp, grid, st) != cudaSuccess) return MOE_ERR_CUDA;
+    return MOE_OK;
+}
+
+moe_status moe_step_host(moe_ctx *ctx, const float *logits_host, const void *x_host, int32_t T,
+                         const moe_dispatch_out *out, float *logits_dev, void *x_dev, void *y_dev,
+                         void *y_host, void *cuda_stream)
+{
+    if (!ctx || !out || T < 0) return MOE_ERR_INVALID_ARG;
+    if (T > ctx->cfg.max_tokens) return MOE_ERR_CAPACITY;
+    if (T > 0 && (!logits_host || !x_host || !logits_dev || !x_dev || !y_dev || !y_host))
+        return MOE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const Derived &d = ctx->d;
+    if (T > 0) {
+        if (cudaMemcpyAsync(logits_dev, logits_host, (size_t)T * d.E * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+            cudaMemcpyAsync(x_dev, x_host, (size_t)T * d.H * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return MOE_ERR_CUDA;
+    }
+    moe_status ms = moe_dispatch(ctx, logits_dev, x_dev, T, out, cuda_stream);
+    if (ms != MOE_OK) return ms;
+    ms = moe_combine(ctx, out->send_buf, T, y_dev, cuda_stream);
+    if (ms != MOE_OK) return ms;
+    if (T > 0 && cudaMemcpyAsync(y_host, y_dev, (size_t)T * d.H * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return MOE_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return MOE_ERR_CUDA;
+    return MOE_OK;
+}
+
+moe_status moe_set_timing_event(moe_ctx *ctx, void *cuda_event)
+{
+    if (!ctx) return MOE_ERR_INVALID_ARG;
+    ctx->timing_event = static_cast<cudaEvent_t>(cuda_event);
+    return MOE_OK;
+}
+
+moe_status moe_get_device_status(moe_ctx *ctx, int32_t *code)
+{
+    if (!ctx || !code) return MOE_ERR_INVALID_ARG;
+    moe::Control c;
+    if (cudaDeviceSynchronize() != cudaSuccess ||
+        cudaMemcpy(&c, ctx->d_ctl, sizeof(c), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return MOE_ERR_CUDA;
+    *code = c.status;
+    if (c.status != kDevOk) {
+        // stale look-back descriptors carry the failed step's epoch: move past it
+        unsigned next = c.epoch + 1u;
+        const moe::Control fresh = {0u, next ? next : 1u, kDevOk, 0};
+        if (cudaMemcpy(ctx->d_ctl, &fresh, sizeof(fresh), cudaMemcpyHostToDevice) != cudaSuccess)
+            return MOE_ERR_CUDA;
+    }
+    return MOE_OK;
+}
+
+moe_status moe_route_destroy(moe_ctx *ctx)
+{
+    if (!ctx) return MOE_OK;
+    cudaDeviceSynchronize();
+    free_ctx(ctx);
+    return MOE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,206 @@
+// K_scatter: finish the permutation (dst_row, src_index) and copy every token's
+// bf16 row into its k rows of the expert-contiguous send buffer.  Each x row is
+// read from HBM once and written k times: (1 + k) rows of traffic per token.
+//
+// Two implementations of the same copy:
+//   k_scatter_vec  — 128-bit loads/stores, a warp per (token, 2 KB column chunk).
+//   k_scatter_bulk — the row is staged in shared memory by one bulk async copy
+//                    (TMA engine, mbarrier completion) and leaves as k bulk
+//                    stores; a multi-stage ring keeps loads ahead of stores.
+#pragma once
+
+#include "device_utils.cuh"
+
+namespace moe {
+
+struct ScatterParams {
+    const uint4 *x;               // [T, H/8] 16-byte units
+    uint4 *send;                  // [T*k, H/8]
+    int T, k, hv;                 // hv = H/8 (uint4 per row)
+    const int32_t *topk_slot;     // [T,k]
+    const int32_t *slot_offsets;  // [P+1]
+    const int32_t *pos_in_slot;   // [T*k] stable rank inside the slot (routing kernel's scratch)
+    int32_t *dst_row;             // out: send-buffer row of assignment i
+    int32_t *src_index;           // out: inverse permutation
+    Control *ctl;
+};
+
+constexpr int kScatterThreads = 256;
+constexpr int kScatterUnroll = 4;                       // 16-byte loads in flight per lane
+constexpr int kScatterChunk = 32 * kScatterUnroll;      // uint4 per work item (2 KB)
+
+// a9 (final step): row = slot_offsets[slot] + rank inside the slot.  Lane j < k
+// owns assignment t*k + j.  Only read-only inputs are used, so any number of
+// warps may resolve the same token; exactly one of them writes the result.
+__device__ __forceinline__ int resolve_row(const ScatterParams &p, int t, int lane, bool write_back)
+{
+    int row = 0;
+    if (lane < p.k) {
+        const size_t i = (size_t)t * p.k + lane;
+        const int slot = __ldg(p.topk_slot + i);
+        row = __ldg(p.slot_offsets + slot) + __ldg(p.pos_in_slot + i);
+        if (write_back) {
+            p.dst_row[i] = row;
+            p.src_index[row] = (int)i;
+        }
+    }
+    return row;
+}
+
+__global__ void __launch_bounds__(kScatterThreads) k_scatter_vec(ScatterParams p)
+{
+    const unsigned full = 0xffffffffu;
+    const int lane = lane_id();
+    const int chunks = (p.hv + kScatterChunk - 1) / kScatterChunk;
+    const long long items = (long long)p.T * chunks;
+    const long long warp0 = (long long)blockIdx.x * (kScatterThreads / 32) + (threadIdx.x >> 5);
+    const long long nwarps = (long long)gridDim.x * (kScatterThreads / 32);
+
+    for (long long it = warp0; it < items; it += nwarps) {
+        const int t = (int)(it / chunks);
+        const int c0 = (int)(it % chunks) * kScatterChunk + lane;
+        const uint4 *src = p.x + (size_t)t * p.hv;
+        uint4 v[kScatterUnroll];
+#pragma unroll
+        for (int u = 0; u < kScatterUnroll; ++u)
+            if (c0 + 32 * u < p.hv) v[u] = ld_stream_v4(src + c0 + 32 * u);
+        const int row = resolve_row(p, t, lane, it % chunks == 0);
+        for (int j = 0; j < p.k; ++j) {
+            const int r = __shfl_sync(full, row, j);
+            uint4 *dst = p.send + (size_t)r * p.hv;
+#pragma unroll
+            for (int u = 0; u < kScatterUnroll; ++u)
+                if (c0 + 32 * u < p.hv) st_stream_v4(dst + c0 + 32 * u, v[u]);
+        }
+    }
+}
+
+// --------------------------- bulk-copy variant -----------------------------
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p)
+{
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, unsigned count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count));
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, unsigned bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)),
+                 "r"(bytes)
+                 : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, unsigned parity)
+{
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_addr(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// global -> shared bulk copy, completion counted in bytes on an mbarrier
+__device__ __forceinline__ void bulk_load(void *smem_dst, const void *gsrc, unsigned bytes,
+                                          uint64_t *bar)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::
+            "r"(smem_addr(smem_dst)),
+        "l"(gsrc), "r"(bytes), "r"(smem_addr(bar))
+        : "memory");
+}
+
+// shared -> global bulk copy, tracked by the issuing thread's bulk async-group
+__device__ __forceinline__ void bulk_store(void *gdst, const void *smem_src, unsigned bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst),
+                 "r"(smem_addr(smem_src)), "r"(bytes)
+                 : "memory");
+}
+
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+
+template <int N>
+__device__ __forceinline__ void bulk_wait_read()
+{
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+constexpr int kBulkThreads = 32;   // one warp per CTA; several CTAs share an SM
+
+// One warp per CTA walks tokens blockIdx.x, blockIdx.x + gridDim.x, ...  Stage s
+// of the ring holds one row.  Lane 0 issues the loads; lane j < k issues the
+// store of row j, so the k stores of a token leave from k different threads.
+// Before a stage is refilled every lane waits until its own earlier stores have
+// finished READING shared memory (they may still be in flight to HBM).
+__global__ void __launch_bounds__(kBulkThreads) k_scatter_bulk(ScatterParams p, int stages)
+{
+    extern __shared__ __align__(128) unsigned char ring[];
+    __shared__ __align__(8) uint64_t full_bar[8];
+    const int lane = lane_id();
+    const unsigned row_bytes = (unsigned)p.hv * 16u;
+    const unsigned stage_bytes = (row_bytes + 127u) & ~127u;
+
+    if (lane == 0) {
+        for (int s = 0; s < stages; ++s) mbar_init(&full_bar[s], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+
+    const int first = blockIdx.x, step = gridDim.x;
+    const int n_mine = (first < p.T) ? (p.T - first + step - 1) / step : 0;
+
+    // prologue: fill the ring except one stage
+    if (lane == 0) {
+        for (int n = 0; n < min(stages - 1, n_mine); ++n) {
+            mbar_expect_tx(&full_bar[n], row_bytes);
+            bulk_load(ring + (size_t)n * stage_bytes,
+                      p.x + (size_t)(first + (size_t)n * step) * p.hv, row_bytes, &full_bar[n]);
+        }
+    }
+    bool ok = true;
+    for (int n = 0; n < n_mine && ok; ++n) {
+        const int t = first + n * step;
+        const int s = n % stages;
+        const int row = resolve_row(p, t, lane, true);
+        // refill the stage freed in the previous iteration with token n + stages - 1
+        const int n_next = n + stages - 1;
+        if (n_next < n_mine) {
+            if (n > 0) bulk_wait_read<0>();      // my store of iteration n-1 has left shared memory
+            __syncwarp();
+            if (lane == 0) {
+                const int sn = n_next % stages;
+                mbar_expect_tx(&full_bar[sn], row_bytes);
+                bulk_load(ring + (size_t)sn * stage_bytes,
+                          p.x + (size_t)(first + (size_t)n_next * step) * p.hv, row_bytes,
+                          &full_bar[sn]);
+            }
+        }
+        // wait for this token's row
+        const unsigned parity = (unsigned)(n / stages) & 1u;
+        unsigned spins = 0;
+        while (!mbar_try_wait(&full_bar[s], parity)) {
+            if (++spins > kSpinLimit) { ok = false; break; }
+        }
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        if (lane < p.k) {
+            bulk_store(p.send + (size_t)row * p.hv, ring + (size_t)s * stage_bytes, row_bytes);
+            bulk_commit();
+        }
+    }
+    if (!ok && lane == 0) report_status(p.ctl, kDevTimeout);
+    bulk_wait_all();   // nothing of this CTA may still read the ring or write HBM at exit
+}
+
+}  // namespace moe

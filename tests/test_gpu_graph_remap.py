@@ -1,0 +1,154 @@
+"""Recovery on the GPU: a remap rewrites only the rank bitmap / replica table in
+device memory, so one captured CUDA graph of dispatch + combine stays valid
+across failures (the paper recompiles its graph instead, Sec. 3.6)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2602_21140_b200 import binding as B
+from paper_2602_21140_b200 import workloads as W
+from gpu_util import assert_y_close, bf16_bits, check_dispatch, make_router, to_dev
+from util import oracle_cfg
+
+pytestmark = pytest.mark.gpu
+
+
+def _capture(router, logits, x, T):
+    out = router.alloc_outputs(T)
+    y = torch.empty((T, router.cfg.hidden), dtype=torch.bfloat16, device="cuda")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        for _ in range(2):                                   # warm-up outside capture
+            router.dispatch(logits, x, out)
+            router.combine(out.send_buf, T, y)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        router.dispatch(logits, x, out)
+        router.combine(out.send_buf, T, y)
+    return graph, out, y
+
+
+def _oracle_step(wl, inp, failed, s2e=None):
+    s2e = inp["slot_to_expert"] if s2e is None else s2e
+    bias = inp["bias"] if wl.score_func == W.SIGMOID else None
+    ref = oracle.dispatch(oracle_cfg(wl), s2e, failed, bias, inp["logits"], inp["x"])
+    ref["y"] = oracle.combine(ref["send_buf"], ref["dst_row"], ref["topk_weights"], ref["topk_slot"],
+                              inp["slot_scale"])
+    return ref
+
+
+@pytest.mark.parametrize("name", ["tiny", "dsv3", "kimi"])
+def test_one_graph_survives_a_sweep_of_failures(name):
+    wl = W.WORKLOADS[name]
+    T, H = min(wl.T, 600), min(wl.H, 512)
+    inp = W.make_inputs(wl, T=T, H=H)
+    router = make_router(wl, inp, max_tokens=T, hidden=H)
+    logits, x = to_dev(inp["logits"]), to_dev(inp["x"], torch.bfloat16)
+    graph, out, y = _capture(router, logits, x, T)
+    sets = list(wl.failure_sets) + [()]
+    for failed in sets:
+        router.set_failed_ranks(failed)          # between replays, on the replay stream
+        graph.replay()                           # the same executable graph every time
+        torch.cuda.synchronize()
+        ref = _oracle_step(wl, inp, failed)
+        check_dispatch(out, ref)
+        assert_y_close(bf16_bits(y), ref["y"])
+        if failed:
+            assert not np.isin(out.topk_slot.cpu().numpy() // wl.S, list(failed)).any()
+            assert int(out.rank_counts.cpu()[list(failed)].sum()) == 0
+    assert router.device_status() == 0
+    router.close()
+
+
+def test_replays_are_bit_identical():
+    wl = W.WORKLOADS["dsv3"]
+    T = 2048
+    inp = W.make_inputs(wl, T=T, H=1024)
+    router = make_router(wl, inp, max_tokens=T, hidden=1024)
+    router.set_failed_ranks((7,))
+    logits, x = to_dev(inp["logits"]), to_dev(inp["x"], torch.bfloat16)
+    graph, out, y = _capture(router, logits, x, T)
+    graph.replay()
+    torch.cuda.synchronize()
+    first = {f: getattr(out, f).clone() for f in out.__dataclass_fields__}
+    y0 = y.clone()
+    for _ in range(20):
+        graph.replay()
+    torch.cuda.synchronize()
+    for f, v in first.items():
+        assert torch.equal(getattr(out, f).view(torch.int32) if v.dtype == torch.float32 else getattr(out, f),
+                           v.view(torch.int32) if v.dtype == torch.float32 else v), f
+    assert torch.equal(y.view(torch.int16), y0.view(torch.int16))
+    router.close()
+
+
+def test_rejected_remap_leaves_device_state_untouched():
+    wl = W.WORKLOADS["mixtral"]
+    inp = W.make_inputs(wl, T=200, H=128)
+    router = make_router(wl, inp, max_tokens=200, hidden=128)
+    router.set_failed_ranks((3,))
+    logits, x = to_dev(inp["logits"]), to_dev(inp["x"], torch.bfloat16)
+    with pytest.raises(B.MoeError) as e:
+        router.set_failed_ranks((0, 1, 2, 3, 4, 5, 6))     # one expert left < k = 2
+    assert e.value.status == B.MOE_ERR_INSUFFICIENT_EXPERTS
+    with pytest.raises(B.MoeError) as e:
+        router.set_failed_ranks((8,))
+    assert e.value.status == B.MOE_ERR_INVALID_ARG
+    out = router.dispatch(logits, x)
+    torch.cuda.synchronize()
+    check_dispatch(out, _oracle_step(wl, inp, (3,)))
+    router.close()
+
+
+def test_failed_ranks_equal_emptied_slots_in_the_map():
+    wl = W.WORKLOADS["dsv3"]
+    inp = W.make_inputs(wl, T=300, H=128)
+    logits, x = to_dev(inp["logits"]), to_dev(inp["x"], torch.bfloat16)
+    failed = (7, 20)
+    a = make_router(wl, inp, max_tokens=300, hidden=128)
+    a.set_failed_ranks(failed)
+    out_a = a.dispatch(logits, x)
+    b = make_router(wl, inp, max_tokens=300, hidden=128)
+    s2e = inp["slot_to_expert"].copy()
+    for r in failed:
+        s2e[r * wl.S:(r + 1) * wl.S] = -1
+    b.update_replica_map(s2e)
+    out_b = b.dispatch(logits, x)
+    torch.cuda.synchronize()
+    for f in out_a.__dataclass_fields__:
+        assert torch.equal(getattr(out_a, f), getattr(out_b, f)), f
+    check_dispatch(out_b, _oracle_step(wl, inp, (), s2e))
+    # moving a replica: expert 0 gains a copy on the last rank's spare slot if it is empty
+    a.close(); b.close()
+
+
+def test_many_back_to_back_remaps_keep_order():
+    wl = W.WORKLOADS["kimi"]
+    inp = W.make_inputs(wl, T=128, H=64)
+    router = make_router(wl, inp, max_tokens=128, hidden=64)
+    logits, x = to_dev(inp["logits"]), to_dev(inp["x"], torch.bfloat16)
+    rng = np.random.default_rng(2)
+    last = ()
+    for i in range(50):                          # more than the staging ring holds
+        last = tuple(int(r) for r in rng.choice(wl.R, int(rng.integers(0, 6)), replace=False))
+        router.set_failed_ranks(last)
+    out = router.dispatch(logits, x)
+    torch.cuda.synchronize()
+    check_dispatch(out, _oracle_step(wl, inp, last))
+    router.close()
+
+
+def test_remap_while_capturing_is_refused():
+    wl = W.WORKLOADS["tiny"]
+    inp = W.make_inputs(wl)
+    router = make_router(wl, inp, max_tokens=wl.T)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        st = B.moe_set_failed_ranks(router._ctx, [2], torch.cuda.current_stream().cuda_stream)
+        torch.zeros(1, device="cuda").add_(1)
+    assert st == B.MOE_ERR_INVALID_ARG
+    router.close()
