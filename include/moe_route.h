@@ -199,6 +199,43 @@ moe_status moe_plan_routing_state(const moe_config *cfg, const int32_t *slot_to_
                                   uint32_t *rank_alive, int32_t *replica_table,
                                   int32_t *n_available);
 
+/*
+ * moe_permute_static — the count / prefix-scan / stable-permutation step of a
+ * dispatch, for callers that cannot allocate device memory.  (The paper has no
+ * counterpart; this exists for deployment reasons only.)
+ *
+ * Who needs it: a process that cannot call cudaMalloc while it is serving —
+ * typically an inference engine that reserved all of HBM for its own pool at
+ * start-up, so that any later allocation fails, or code running where the CUDA
+ * runtime does not permit allocation.  Such a caller cannot create a context
+ * with moe_route_init (which allocates scan scratch), but it can still hand
+ * pre-existing buffers to this function.  The function allocates nothing, on
+ * the host or the device: its scratch is a fixed 512 KiB array inside the
+ * library's device image, present on every GPU that loads the library until
+ * the process exits.
+ *
+ *   topk_slot    device [n_assign] i32  physical slot of each assignment i, in [0, P);
+ *                                       entries outside that range are ignored
+ *   slot_counts  device [P]   i32 out   slot_offsets device [P+1] i32 out
+ *   rank_counts  device [R]   i32 out   rank_offsets device [R+1] i32 out
+ *   dst_row      device [n_assign] i32 out   src_index device [n_assign] i32 out
+ * with P = num_ranks * slots_per_rank; meanings as in moe_dispatch_out.
+ *
+ * Limits: P <= 512 and n_assign <= 262144; anything larger returns
+ * MOE_ERR_CAPACITY and launches nothing.  n_assign = 0 writes zero counts.
+ * The first call on each device looks up the scratch array's device address
+ * (one runtime query, no allocation); make that first call before starting any
+ * stream capture.  All calls on a device share the one array: the function
+ * rewrites every word it reads, so leftovers of earlier calls are harmless,
+ * but two calls that overlap on the GPU (different streams without ordering)
+ * race on it.  Work is enqueued on `cuda_stream`; the call does not wait.
+ */
+moe_status moe_permute_static(const int32_t *topk_slot, int32_t n_assign,
+                              int32_t num_ranks, int32_t slots_per_rank,
+                              int32_t *slot_counts, int32_t *slot_offsets,
+                              int32_t *rank_counts, int32_t *rank_offsets,
+                              int32_t *dst_row, int32_t *src_index, void *cuda_stream);
+
 /* Device bytes a context for `cfg` allocates (0 if cfg is invalid). */
 size_t moe_workspace_bytes(const moe_config *cfg);
 

@@ -37,7 +37,7 @@ MOE_SCORE_SIGMOID = 1
 EXPORTED_SYMBOLS = (
     "moe_route_init", "moe_set_failed_ranks", "moe_update_replica_map", "moe_dispatch",
     "moe_combine", "moe_step_host", "moe_set_timing_event", "moe_get_device_status", "moe_plan_routing_state",
-    "moe_workspace_bytes", "moe_route_destroy", "moe_status_string",
+    "moe_workspace_bytes", "moe_route_destroy", "moe_status_string", "moe_permute_static",
 )
 
 
@@ -100,6 +100,8 @@ def _lib():
         lib.moe_workspace_bytes.argtypes = [ctypes.POINTER(moe_config)]
         lib.moe_route_destroy.restype = ctypes.c_int
         lib.moe_route_destroy.argtypes = [vp]
+        lib.moe_permute_static.restype = ctypes.c_int
+        lib.moe_permute_static.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
         lib.moe_status_string.restype = ctypes.c_char_p
         lib.moe_status_string.argtypes = [ctypes.c_int]
         _lib_handle = lib
@@ -197,6 +199,20 @@ def moe_get_device_status(ctx):
     code = ctypes.c_int32(0)
     st = _lib().moe_get_device_status(ctx, ctypes.byref(code))
     return st, int(code.value)
+
+
+def moe_permute_static(topk_slot_ptr: int, n_assign: int, num_ranks: int, slots_per_rank: int,
+                       slot_counts_ptr: int, slot_offsets_ptr: int, rank_counts_ptr: int,
+                       rank_offsets_ptr: int, dst_row_ptr: int, src_index_ptr: int,
+                       cuda_stream: int = 0) -> int:
+    """Count / scan / stable permutation from caller-owned device buffers, using only the
+    library's built-in scratch array: for callers that are not able to allocate device
+    memory (see include/moe_route.h).  All pointer arguments are raw device addresses."""
+    vp = ctypes.c_void_p
+    return _lib().moe_permute_static(vp(topk_slot_ptr), n_assign, num_ranks, slots_per_rank,
+                                     vp(slot_counts_ptr), vp(slot_offsets_ptr), vp(rank_counts_ptr),
+                                     vp(rank_offsets_ptr), vp(dst_row_ptr), vp(src_index_ptr),
+                                     vp(cuda_stream))
 
 
 def moe_route_destroy(ctx) -> int:
