@@ -139,7 +139,9 @@ def time_oracle(wl, inp, failed, budget_s=12.0, t_probe=256):
     t0 = time.perf_counter()
     oracle_step(wl, inp, failed, t_probe)
     per_tok = (time.perf_counter() - t0) / t_probe
-    T_s = int(max(64, min(wl.T, budget_s / 3 / per_tok)))
+    n_tok = inp["logits"].shape[0]
+    t_probe = min(t_probe, n_tok)
+    T_s = int(max(min(64, n_tok), min(n_tok, budget_s / 3 / per_tok)))
     n, t_start = 0, time.perf_counter()
     while n < 3 or (time.perf_counter() - t_start < budget_s and n < 50):
         oracle_step(wl, inp, failed, T_s)
@@ -148,7 +150,7 @@ def time_oracle(wl, inp, failed, budget_s=12.0, t_probe=256):
             break
     dt = time.perf_counter() - t_start
     return {"value": T_s * n / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": f"{n} dispatch+combine steps over the first {T_s} of {wl.T} tokens, {dt:.1f} s, single thread"}
+            "sample": f"{n} dispatch+combine steps over the first {T_s} of {n_tok} tokens, {dt:.1f} s, single thread"}
 
 
 def run_reference(args):
@@ -223,10 +225,11 @@ def run_ours(args):
 
     wl = W.WORKLOADS[args.workload]
     failed = wl.failure_sets[args.failure_set]
-    T, K, Wm = wl.T, args.steps, args.warmup
-    inp = W.make_inputs(wl, seed=shard_seed(wl.seed, rank))
+    T, K, Wm = (args.tokens or wl.T), args.steps, args.warmup
+    inp = W.make_inputs(wl, T=T, seed=shard_seed(wl.seed, rank))
     bias = inp["bias"] if wl.score_func == W.SIGMOID else None
-    router = B.MoeRouter(B.config_for_workload(wl), inp["slot_to_expert"], bias, inp["slot_scale"], device=dev)
+    router = B.MoeRouter(B.config_for_workload(wl, max_tokens=T), inp["slot_to_expert"], bias,
+                         inp["slot_scale"], device=dev)
     router.set_failed_ranks(failed)
 
     lg_h = torch.from_numpy(inp["logits"]).pin_memory()
@@ -239,6 +242,22 @@ def run_ours(args):
     stream = torch.cuda.Stream(device=dev)
     stream.wait_stream(torch.cuda.current_stream())
     launches = 0
+    if args.quick:
+        # profiling aid: a few eager steps and nothing else, so that a profiler capture stays short
+        with torch.cuda.stream(stream):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            for i in range(Wm + K):
+                if i == Wm:
+                    e0.record(stream)
+                router.dispatch(logits, x, out)
+                router.combine(out.send_buf, T, y)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            assert router.device_status() == 0
+        print(json.dumps({"quick": True, "workload": workload_name(wl, failed), "tokens": T, "steps": K,
+                          "ms_per_step": e0.elapsed_time(e1) / max(K, 1)}))
+        router.close()
+        return
     with torch.cuda.stream(stream):
         for _ in range(max(Wm, 3)):
             router.dispatch(logits, x, out)
@@ -387,6 +406,8 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default="dsv3")
     ap.add_argument("--failure-set", type=int, default=1, help="index into the workload's failure sets")
+    ap.add_argument("--tokens", type=int, default=0, help="override T (profiling captures on a smaller case)")
+    ap.add_argument("--quick", action="store_true", help="a few eager steps only (for profiler captures)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

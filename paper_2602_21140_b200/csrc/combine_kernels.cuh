@@ -107,4 +107,146 @@ __global__ void __launch_bounds__(kCombineThreads) k_combine_vec(CombineParams p
     }
 }
 
+// ------------------------------ bulk-copy variant ---------------------------
+// Each warp owns a ring of `stages` shared-memory stages; a stage holds the same
+// column chunk (32*U 16-byte units) of the k rows of one token.  Lane j < k asks
+// the TMA engine for row j's chunk (one bulk copy each, all counted on the
+// stage's mbarrier), so many kilobytes per warp are in flight without holding
+// registers, and the warp only touches a stage once it has landed.  Items
+// (token, chunk) are dealt to warps in contiguous runs, so a warp re-reads the
+// row indices and coefficients only when it moves to the next token, and those
+// are fetched one token ahead.
+constexpr int kCombineBulkMaxWarps = 8;   // warps per CTA (blockDim.x / 32), each with its own ring
+
+struct CombineIssue {   // per-lane state of the issuing side (lane j < k)
+    int token;
+    int row, row_next;
+    float coef, coef_next;
+};
+
+__device__ __forceinline__ void combine_fetch_index(const CombineParams &p, int t, int lane, int &row,
+                                                    float &coef)
+{
+    row = 0; coef = 0.0f;
+    if (lane < p.k && t < p.T) {
+        const size_t i = (size_t)t * p.k + lane;
+        row = __ldg(p.dst_row + i);
+        coef = __fmul_rn(__ldg(p.topk_weights + i), __ldg(p.slot_scale + __ldg(p.topk_slot + i)));
+    }
+}
+
+template <int U>
+__global__ void __launch_bounds__(kCombineBulkMaxWarps * 32) k_combine_bulk(CombineParams p, int stages,
+                                                                         Control *ctl)
+{
+    extern __shared__ __align__(128) unsigned char dyn[];
+    constexpr int kChunkV = 32 * U;                       // 16-byte units per row chunk
+    constexpr unsigned kChunkBytes = kChunkV * 16u;
+    const int lane = lane_id(), warp = threadIdx.x >> 5;
+    const int kCombineBulkWarps = blockDim.x >> 5;
+    const int k = p.k;
+    const unsigned stage_bytes = (unsigned)k * kChunkBytes;
+    // per-warp carve-up: [stages][k][chunk] data, then [stages][k] coefficients, then barriers
+    const size_t warp_bytes = (size_t)stages * stage_bytes;
+    unsigned char *ring = dyn + (size_t)warp * warp_bytes;
+    float *coefs = reinterpret_cast<float *>(dyn + (size_t)kCombineBulkWarps * warp_bytes) +
+                   (size_t)warp * stages * k;
+    uint64_t *full = reinterpret_cast<uint64_t *>(
+                         dyn + (size_t)kCombineBulkWarps * warp_bytes +
+                         (((size_t)kCombineBulkWarps * stages * k * 4 + 7) & ~(size_t)7)) +
+                     (size_t)warp * stages;
+
+    if (lane == 0) {
+        for (int s = 0; s < stages; ++s) mbar_init(&full[s], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+
+    const int chunks = (p.hv + kChunkV - 1) / kChunkV;
+    const long long items = (long long)p.T * chunks;
+    const long long nwarps = (long long)gridDim.x * kCombineBulkWarps;
+    const long long wid = (long long)blockIdx.x * kCombineBulkWarps + warp;
+    const long long per = items / nwarps, extra = items % nwarps;      // contiguous, balanced runs
+    const long long first = wid * per + (wid < extra ? wid : extra);
+    const int n_mine = (int)(per + (wid < extra ? 1 : 0));
+    if (n_mine == 0) return;
+
+    CombineIssue is;
+    is.token = (int)(first / chunks);
+    combine_fetch_index(p, is.token, lane, is.row, is.coef);
+    combine_fetch_index(p, is.token + 1, lane, is.row_next, is.coef_next);
+
+    auto issue = [&](int n) {
+        const long long item = first + n;
+        const int t = (int)(item / chunks);
+        const int c0 = (int)(item % chunks) * kChunkV;
+        if (t != is.token) {                               // moved on: take the prefetched indices
+            is.token = t; is.row = is.row_next; is.coef = is.coef_next;
+            combine_fetch_index(p, t + 1, lane, is.row_next, is.coef_next);
+        }
+        const int s = n % stages;
+        const unsigned bytes = (unsigned)min(kChunkV, p.hv - c0) * 16u;
+        if (lane == 0) mbar_expect_tx(&full[s], bytes * (unsigned)k);
+        __syncwarp();
+        if (lane < k) {
+            coefs[s * k + lane] = is.coef;
+            bulk_load(ring + (size_t)s * stage_bytes + (size_t)lane * kChunkBytes,
+                      p.buf + (size_t)is.row * p.hv + c0, bytes, &full[s]);
+        }
+    };
+
+    for (int n = 0; n < min(stages - 1, n_mine); ++n) issue(n);
+
+    bool ok = true;
+    int n = 0;
+    for (; n < n_mine; ++n) {
+        if (n + stages - 1 < n_mine) issue(n + stages - 1);   // refills the stage consumed at n-1
+        const int s = n % stages;
+        const unsigned parity = (unsigned)(n / stages) & 1u;
+        unsigned spins = 0;
+        while (!mbar_try_wait(&full[s], parity)) {
+            if (++spins > kSpinLimit) { ok = false; break; }
+        }
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        __syncwarp();                                      // coefficients written at issue are visible
+        const long long item = first + n;
+        const int t = (int)(item / chunks);
+        const int c0 = (int)(item % chunks) * kChunkV + lane;
+        float acc[U][8];
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+#pragma unroll
+            for (int q = 0; q < 8; ++q) acc[u][q] = 0.0f;
+        const uint4 *st = reinterpret_cast<const uint4 *>(ring + (size_t)s * stage_bytes);
+        for (int j = 0; j < k; ++j) {
+            const float c = coefs[s * k + j];
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                if (c0 + 32 * u < p.hv) fma_bf16x8(acc[u], st[j * kChunkV + lane + 32 * u], c);
+        }
+        uint4 *dst = p.y + (size_t)t * p.hv;
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (c0 + 32 * u < p.hv) st_stream_v4(dst + c0 + 32 * u, pack_bf16x8(acc[u]));
+        __syncwarp();                                      // every lane is done reading stage s
+    }
+    if (!ok) {
+        if (lane == 0) report_status(ctl, kDevTimeout);
+        // copies issued for items n .. n+stages-2 may still be landing in this CTA's shared
+        // memory: give each a bounded chance to finish before the memory is released
+        for (int m = n; m < min(n_mine, n + stages - 1); ++m) {
+            unsigned spins = 0;
+            while (!mbar_try_wait(&full[m % stages], (unsigned)(m / stages) & 1u) && ++spins < kSpinLimit) {}
+        }
+    }
+}
+
+__host__ __device__ inline size_t combine_bulk_smem(int stages, int k, int U, int kCombineBulkWarps)
+{
+    const size_t warp_bytes = (size_t)stages * k * 32 * U * 16;
+    const size_t coef_bytes = ((size_t)kCombineBulkWarps * stages * k * 4 + 7) & ~(size_t)7;
+    return kCombineBulkWarps * warp_bytes + coef_bytes + (size_t)kCombineBulkWarps * stages * 8;
+}
+
 }  // namespace moe

@@ -31,6 +31,7 @@ constexpr size_t kMaxSmem = 227 * 1024;
 struct Derived {
     int E, k, H, P, R, S, max_rep;
     int epl;               // experts per lane in the routing warp
+    int lpt;               // lanes per token in the routing warp (8 or 16)
     int lanes_per_group;   // lanes holding one expert group (power of two), 0 if ungrouped
     int group_m;           // keys summed into a group score
     int rank_words;        // words of the rank bitmap
@@ -58,30 +59,42 @@ bool derive(const moe_config *c, Derived *d)
     d->E = c->num_experts; d->k = c->top_k; d->H = c->hidden; d->P = (int)P;
     d->R = c->num_ranks; d->S = c->slots_per_rank; d->max_rep = c->max_replicas;
     d->lanes_per_group = 0; d->group_m = 1;
-    static const int kEpl[] = {1, 2, 3, 4, 5, 6, 7, 8, 10, 12, 16};
-    d->epl = 0;
+    // lanes per token (8 or 16, at least k) and experts per lane: the smallest pair that
+    // covers E and, with groups, puts every group on a power-of-two run of whole lanes
+    static const int kEpl[] = {1, 2, 3, 4, 5, 6, 8, 10, 12, 16, 20, 24, 32};
+    static const int kLpt[] = {8, 16};
+    d->epl = 0; d->lpt = 0;
     if (c->n_group > 1) {
         if (c->topk_group < 1 || c->topk_group > c->n_group) return false;
         if (d->E % c->n_group != 0 || d->k % c->topk_group != 0) return false;
         d->group_m = d->k / c->topk_group;
         if (d->group_m != 1 && d->group_m != 2) return false;
-        const int per = d->E / c->n_group;
+    } else if (c->n_group != 1) {
+        return false;
+    }
+    for (int lpt : kLpt) {
+        if (d->epl || d->k > lpt) continue;
         for (int epl : kEpl) {
-            if (32 * epl < d->E || per % epl != 0) continue;
-            const int lpg = per / epl;
-            if (!is_pow2(lpg) || lpg * c->n_group > 32) continue;
-            d->epl = epl; d->lanes_per_group = lpg;
+            if (lpt * epl < d->E) continue;
+            if (c->n_group > 1) {
+                const int per = d->E / c->n_group;
+                if (per % epl != 0) continue;
+                const int lpg = per / epl;
+                if (!is_pow2(lpg) || lpg * c->n_group > lpt) continue;
+                d->lanes_per_group = lpg;
+            }
+            d->epl = epl; d->lpt = lpt;
             break;
         }
-    } else {
-        if (c->n_group != 1) return false;
-        for (int epl : kEpl)
-            if (32 * epl >= d->E) { d->epl = epl; break; }
     }
     if (d->epl == 0) return false;
     d->rank_words = (d->R + 31) / 32;
     d->state_words = kStateHeaderWords + d->rank_words + d->E * d->max_rep;
+    // routing tile: a power of two, grown with max_tokens so that a step has <= 128 tiles
     d->tokens_per_block = 32;
+    while ((c->max_tokens + d->tokens_per_block - 1) / d->tokens_per_block > kMaxRouteTiles)
+        d->tokens_per_block *= 2;
+    if (d->tokens_per_block > 2048) return false;      // max_tokens <= 262144
     if (route_smem_bytes(d->E, d->max_rep, d->tokens_per_block, d->k, d->P) > kMaxSmem - 1024)
         return false;
     return true;
@@ -171,6 +184,9 @@ struct moe_ctx {
     int scatter_impl;      // 0 = vector, 1 = bulk copies
     int bulk_stages, bulk_ctas_per_sm;
     int scatter_blocks_per_sm, combine_blocks_per_sm;
+    int combine_impl;      // 0 = vector loads, 1 = bulk-copy ring
+    int combine_stages, combine_u, combine_ctas_per_sm, combine_warps;
+    size_t combine_smem;
     size_t route_smem;
     // what the latest dispatch wrote, for combine
     const float *last_weights;
@@ -194,33 +210,43 @@ size_t device_bytes_for(const Derived &d, int max_tokens)
     return b;
 }
 
-template <int EPL>
-cudaError_t launch_route_epl(const RouteParams &p, int tiles, size_t smem, cudaStream_t st)
+template <int EPL, int LPT>
+cudaError_t launch_route_t(const RouteParams &p, int tiles, size_t smem, cudaStream_t st)
 {
     if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(k_route<EPL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(k_route<EPL, LPT>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
-    k_route<EPL><<<tiles, kRouteThreads, smem, st>>>(p);
+    k_route<EPL, LPT><<<tiles, kRouteThreads, smem, st>>>(p);
     return cudaGetLastError();
 }
 
-cudaError_t launch_route(int epl, const RouteParams &p, int tiles, size_t smem, cudaStream_t st)
+template <int LPT>
+cudaError_t launch_route_lpt(int epl, const RouteParams &p, int tiles, size_t smem, cudaStream_t st)
 {
     switch (epl) {
-        case 1: return launch_route_epl<1>(p, tiles, smem, st);
-        case 2: return launch_route_epl<2>(p, tiles, smem, st);
-        case 3: return launch_route_epl<3>(p, tiles, smem, st);
-        case 4: return launch_route_epl<4>(p, tiles, smem, st);
-        case 5: return launch_route_epl<5>(p, tiles, smem, st);
-        case 6: return launch_route_epl<6>(p, tiles, smem, st);
-        case 7: return launch_route_epl<7>(p, tiles, smem, st);
-        case 8: return launch_route_epl<8>(p, tiles, smem, st);
-        case 10: return launch_route_epl<10>(p, tiles, smem, st);
-        case 12: return launch_route_epl<12>(p, tiles, smem, st);
-        case 16: return launch_route_epl<16>(p, tiles, smem, st);
+        case 1: return launch_route_t<1, LPT>(p, tiles, smem, st);
+        case 2: return launch_route_t<2, LPT>(p, tiles, smem, st);
+        case 3: return launch_route_t<3, LPT>(p, tiles, smem, st);
+        case 4: return launch_route_t<4, LPT>(p, tiles, smem, st);
+        case 5: return launch_route_t<5, LPT>(p, tiles, smem, st);
+        case 6: return launch_route_t<6, LPT>(p, tiles, smem, st);
+        case 8: return launch_route_t<8, LPT>(p, tiles, smem, st);
+        case 10: return launch_route_t<10, LPT>(p, tiles, smem, st);
+        case 12: return launch_route_t<12, LPT>(p, tiles, smem, st);
+        case 16: return launch_route_t<16, LPT>(p, tiles, smem, st);
+        case 20: return launch_route_t<20, LPT>(p, tiles, smem, st);
+        case 24: return launch_route_t<24, LPT>(p, tiles, smem, st);
+        case 32: return launch_route_t<32, LPT>(p, tiles, smem, st);
     }
+    return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_route(int epl, int lpt, const RouteParams &p, int tiles, size_t smem, cudaStream_t st)
+{
+    if (lpt == 8) return launch_route_lpt<8>(epl, p, tiles, smem, st);
+    if (lpt == 16) return launch_route_lpt<16>(epl, p, tiles, smem, st);
     return cudaErrorInvalidValue;
 }
 
@@ -393,6 +419,26 @@ moe_status moe_route_init(const moe_config *cfg, const int32_t *slot_to_expert, 
                                       (int)ring) == cudaSuccess;
         ctx->scatter_blocks_per_sm = std::max(1, env_int("MOE_SCATTER_BLOCKS_PER_SM", 8));
         ctx->combine_blocks_per_sm = std::max(1, env_int("MOE_COMBINE_BLOCKS_PER_SM", 8));
+        ctx->combine_impl = env_int("MOE_COMBINE_IMPL", 1);
+        ctx->combine_u = env_int("MOE_COMBINE_U", 2);
+        if (ctx->combine_u != 1 && ctx->combine_u != 2 && ctx->combine_u != 4) ctx->combine_u = 2;
+        ctx->combine_warps = std::min(kCombineBulkMaxWarps, std::max(1, env_int("MOE_COMBINE_WARPS", 4)));
+        ctx->combine_stages = std::min(8, std::max(2, env_int("MOE_COMBINE_STAGES", 2)));
+        while (ctx->combine_stages > 2 &&
+               combine_bulk_smem(ctx->combine_stages, d.k, ctx->combine_u, ctx->combine_warps) > kMaxSmem - 1024)
+            --ctx->combine_stages;
+        ctx->combine_smem = combine_bulk_smem(ctx->combine_stages, d.k, ctx->combine_u, ctx->combine_warps);
+        if (ctx->combine_smem > kMaxSmem - 1024) ctx->combine_impl = 0;
+        if (ctx->combine_impl == 1) {
+            const int fit_c = (int)((kMaxSmem - 1024) / (ctx->combine_smem + 1024));
+            ctx->combine_ctas_per_sm = std::max(1, std::min(fit_c, env_int("MOE_COMBINE_CTAS_PER_SM", fit_c)));
+            ok = ok && cudaFuncSetAttribute(k_combine_bulk<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)ctx->combine_smem) == cudaSuccess
+                    && cudaFuncSetAttribute(k_combine_bulk<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)ctx->combine_smem) == cudaSuccess
+                    && cudaFuncSetAttribute(k_combine_bulk<4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)ctx->combine_smem) == cudaSuccess;
+        }
     }
     if (!ok) {
         cudaGetLastError();
@@ -471,7 +517,7 @@ moe_status moe_dispatch(moe_ctx *ctx, const float *logits, const void *x, int32_
     rp.rank_counts = out->rank_counts; rp.rank_offsets = out->rank_offsets;
     rp.desc = ctx->d_desc; rp.ctl = ctx->d_ctl;
     const int tiles = (T + d.tokens_per_block - 1) / d.tokens_per_block;
-    if (launch_route(d.epl, rp, tiles, ctx->route_smem, st) != cudaSuccess) return MOE_ERR_CUDA;
+    if (launch_route(d.epl, d.lpt, rp, tiles, ctx->route_smem, st) != cudaSuccess) return MOE_ERR_CUDA;
     if (ctx->timing_event && cudaEventRecord(ctx->timing_event, st) != cudaSuccess) return MOE_ERR_CUDA;
 
     ScatterParams sp;
@@ -507,6 +553,20 @@ moe_status moe_combine(moe_ctx *ctx, const void *expert_buf, int32_t T, void *y,
     cp.T = T; cp.k = d.k; cp.hv = d.H / 8;
     cp.dst_row = ctx->last_dst_row; cp.topk_weights = ctx->last_weights; cp.topk_slot = ctx->last_slot;
     cp.slot_scale = ctx->d_slot_scale;
+    if (ctx->combine_impl == 1) {
+        const int chunk_v = 32 * ctx->combine_u;
+        const long long items = (long long)T * ((cp.hv + chunk_v - 1) / chunk_v);
+        const int nw = ctx->combine_warps;
+        const long long want = (items + nw - 1) / nw;
+        const int grid = (int)std::min<long long>(want, (long long)ctx->sm_count * ctx->combine_ctas_per_sm);
+        if (ctx->combine_u == 1)
+            k_combine_bulk<1><<<grid, nw * 32, ctx->combine_smem, st>>>(cp, ctx->combine_stages, ctx->d_ctl);
+        else if (ctx->combine_u == 2)
+            k_combine_bulk<2><<<grid, nw * 32, ctx->combine_smem, st>>>(cp, ctx->combine_stages, ctx->d_ctl);
+        else
+            k_combine_bulk<4><<<grid, nw * 32, ctx->combine_smem, st>>>(cp, ctx->combine_stages, ctx->d_ctl);
+        return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+    }
     const int chunks = (cp.hv + kCombineChunk - 1) / kCombineChunk;
     const long long items = (long long)T * chunks;
     const long long want = (items + kCombineThreads / 32 - 1) / (kCombineThreads / 32);

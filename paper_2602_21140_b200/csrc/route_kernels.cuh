@@ -1,20 +1,29 @@
 // K_route: gate, availability mask, group-limited top-k, weight renormalisation,
-// live-replica pick, per-slot histogram, decoupled look-back scan over tiles and
-// the final per-slot / per-rank offsets — one kernel, one pass over the logits.
+// live-replica pick, per-slot histogram, prefix over tiles by aggregate look-back
+// and the final per-slot / per-rank offsets — one kernel, one pass over the logits.
 //
-// Work split: a CTA of 8 warps takes one tile of `tokens_per_block` consecutive
+// Work split: a CTA of 32 warps takes one tile of `tokens_per_block` consecutive
 // tokens (tiles are handed out by an atomic ticket, so every tile a CTA may wait
-// for is already running).  A warp routes one token at a time with the experts
-// laid out contiguously over lanes (lane l holds experts [l*EPL, (l+1)*EPL)),
-// which makes "lower lane" equal "lower expert id" for tie-breaks and puts a
-// whole expert group inside a power-of-two run of lanes.
+// for is already running).  A warp routes 32/LPT tokens at once: a token owns
+// LPT consecutive lanes and lane s of them holds experts [s*EPL, (s+1)*EPL) in
+// registers, which makes "lower lane" equal "lower expert id" for tie-breaks,
+// puts a whole expert group inside a power-of-two run of lanes, and keeps every
+// lane busy in the serial top-k rounds (the kernel is bound by instruction
+// issue, not by memory).
+//
+// Prefix over tiles: the whole problem fits in one wave of CTAs, so all tiles
+// publish at about the same time and a chained look-back (wait for the
+// predecessor's inclusive prefix) would serialise them.  Instead every tile
+// publishes only its own per-slot aggregate and sums the aggregates of ALL
+// earlier tiles with independent, coalesced loads; the host keeps the number
+// of tiles <= 128 by growing the tile with max_tokens, which bounds that traffic.
 #pragma once
 
 #include "device_utils.cuh"
 
 namespace moe {
 
-constexpr int kRouteThreads = 256;
+constexpr int kRouteThreads = 1024;
 constexpr int kRouteWarps = kRouteThreads / 32;
 
 // Routing state blob in device memory (int32 words), rewritten by a remap:
@@ -24,9 +33,8 @@ constexpr int kRouteWarps = kRouteThreads / 32;
 constexpr int kStateHeaderWords = 2;
 
 // Look-back descriptor, one 64-bit word per (tile, slot):
-//   bits 63..32 epoch of the step that wrote it, 31..30 flag, 29..0 count
-constexpr unsigned long long kFlagAggregate = 1ull;   // count of this tile only
-constexpr unsigned long long kFlagInclusive = 2ull;   // count of tiles 0..this
+//   bits 63..32 epoch of the step that wrote it, 31..0 assignments of the tile on the slot
+constexpr int kMaxRouteTiles = 128;
 
 struct RouteParams {
     const float *logits;      // [T,E]
@@ -49,145 +57,137 @@ struct RouteParams {
 __host__ __device__ inline size_t route_smem_bytes(int E, int max_rep, int tokens_per_block, int k,
                                                    int P)
 {
-    size_t words = (size_t)E + (size_t)E * max_rep + 2 * (size_t)tokens_per_block * k +
-                   2 * (size_t)P + (size_t)kRouteWarps * P;
-    return words * sizeof(int32_t);
+    size_t words = (size_t)E + (size_t)E * max_rep + 2 * (size_t)tokens_per_block * k + 2 * (size_t)P;
+    return words * sizeof(int32_t) + (size_t)kRouteWarps * P * sizeof(uint16_t);
 }
 
-// Route one token with the whole warp.  Lane j < k leaves with the j-th chosen
-// expert, its weight and its physical slot.
-template <int EPL>
-__device__ __forceinline__ void route_token(const RouteParams &p, int t, const int32_t *s_nlive,
-                                            const int32_t *s_live, int fallback_expert,
-                                            int &out_id, float &out_w, int &out_slot)
+// Route 32/LPT tokens with one warp.  Lanes [sub*LPT, (sub+1)*LPT) own token
+// t_first + sub.  On return, sub-lane j < k of a token holds its j-th chosen
+// expert, the weight and the physical slot.
+template <int EPL, int LPT>
+__device__ __forceinline__ void route_tokens(const RouteParams &p, int t_first, uint32_t avail_mask,
+                                             const int32_t *s_nlive, const int32_t *s_live,
+                                             int fallback_expert, int &out_id, float &out_w,
+                                             int &out_slot)
 {
     const unsigned full = 0xffffffffu;
     const int lane = lane_id();
+    const int sub = lane / LPT, sl = lane % LPT;
     const int E = p.E;
-    const int e0 = lane * EPL;
+    const int e0 = sl * EPL;
+    const int t = min(t_first + sub, p.T - 1);           // lanes past the end redo the last token
     const float *row = p.logits + (size_t)t * E;
     const float neg_inf = __int_as_float(0xff800000);
+    const bool sigmoid = p.score_func != 0;
 
-    float val[EPL];    // what the weight is made of: logit (softmax) or sigmoid score
-    float key[EPL];    // what selection compares
-
-    // a1 gate scores, a2 availability mask
-    float lg[EPL];
-    if ((EPL % 4 == 0) && (E == 32 * EPL)) {
-        const float4 *row4 = reinterpret_cast<const float4 *>(row + e0);
+    // a1 gate scores, a2 availability mask, and the two best keys of this lane (for a3)
+    uint32_t code[EPL];
+    float h1 = neg_inf, h2 = neg_inf;
 #pragma unroll
-        for (int q = 0; q < EPL / 4; ++q) {
-            float4 v = __ldg(row4 + q);
-            lg[4 * q] = v.x; lg[4 * q + 1] = v.y; lg[4 * q + 2] = v.z; lg[4 * q + 3] = v.w;
-        }
-    } else {
-#pragma unroll
-        for (int q = 0; q < EPL; ++q) lg[q] = (e0 + q < E) ? __ldg(row + e0 + q) : neg_inf;
-    }
-#pragma unroll
-    for (int q = 0; q < EPL; ++q) {
-        const int e = e0 + q;
-        const bool in_range = e < E;
-        float kf;
-        if (p.score_func == 0) {
-            val[q] = lg[q];
-            kf = lg[q];
+    for (int q0 = 0; q0 < EPL; q0 += 4) {
+        float lg[4];
+        if ((EPL % 4 == 0) && (E == LPT * EPL)) {
+            const float4 v = __ldg(reinterpret_cast<const float4 *>(row + e0 + q0));
+            lg[0] = v.x; lg[1] = v.y; lg[2] = v.z; lg[3] = v.w;
         } else {
-            const float s = sigmoid_spec(lg[q]);
-            val[q] = s;
-            kf = __fadd_rn(s, in_range ? __ldg(p.bias + e) : 0.0f);
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                lg[u] = (q0 + u < EPL && e0 + q0 + u < E) ? __ldg(row + e0 + q0 + u) : neg_inf;
         }
-        const bool ok = in_range && (s_nlive[in_range ? e : 0] > 0) && (lg[q] != neg_inf);
-        key[q] = ok ? kf : neg_inf;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int q = q0 + u;
+            if (q < EPL) {
+                float kf = lg[u];
+                if (sigmoid)
+                    kf = __fadd_rn(sigmoid_spec(lg[u]), (e0 + q < E) ? __ldg(p.bias + e0 + q) : 0.0f);
+                const bool ok = ((avail_mask >> q) & 1u) && (lg[u] != neg_inf);
+                kf = ok ? kf : neg_inf;
+                if (kf > h1) { h2 = h1; h1 = kf; }
+                else if (kf > h2) { h2 = kf; }
+                code[q] = key_code(kf);
+            }
+        }
     }
 
     // a3 group-limited selection: score = sum of the (up to) group_m best finite keys
+    bool active = true;
     if (p.n_group > 1) {
-        float h1 = neg_inf, h2 = neg_inf;
-#pragma unroll
-        for (int q = 0; q < EPL; ++q) {
-            const float v = key[q];
-            if (v > h1) { h2 = h1; h1 = v; }
-            else if (v > h2) { h2 = v; }
-        }
         for (int off = 1; off < p.lanes_per_group; off <<= 1) {
-            const float o1 = __shfl_xor_sync(full, h1, off);
-            const float o2 = __shfl_xor_sync(full, h2, off);
+            const float o1 = __shfl_xor_sync(full, h1, off, LPT);
+            const float o2 = __shfl_xor_sync(full, h2, off, LPT);
             const float n1 = fmaxf(h1, o1);
             const float n2 = fmaxf(fminf(h1, o1), fmaxf(h2, o2));
             h1 = n1; h2 = n2;
         }
         const float gscore = (p.group_m == 1 || h2 == neg_inf) ? h1 : __fadd_rn(h1, h2);
-        const int g = lane / p.lanes_per_group;
+        const int g = sl / p.lanes_per_group;
         int rank = 0;
         for (int gp = 0; gp < p.n_group; ++gp) {
-            const float o = __shfl_sync(full, gscore, gp * p.lanes_per_group);
+            const float o = __shfl_sync(full, gscore, gp * p.lanes_per_group, LPT);
             rank += (o > gscore) || (o == gscore && gp < g);
         }
-        const bool keep = (g < p.n_group) && (rank < p.topk_group);
-        if (!keep) {
-#pragma unroll
-            for (int q = 0; q < EPL; ++q) key[q] = neg_inf;
-        }
+        active = (g < p.n_group) && (rank < p.topk_group);
     }
 
-    // a4 top-k: k rounds of warp arg-max over order-preserving integer codes
-    uint32_t code[EPL];
+    // a4 top-k: k rounds of arg-max over order-preserving integer codes
+    uint32_t lbest = 0; int lq = 0;
+    if (active) {
 #pragma unroll
-    for (int q = 0; q < EPL; ++q) code[q] = key_code(key[q]);
-
-    uint32_t lbest = 0; int lq = 0; float lval = 0.0f;
-#pragma unroll
-    for (int q = 0; q < EPL; ++q)
-        if (code[q] > lbest) { lbest = code[q]; lq = q; lval = val[q]; }
-
-    int my_id = fallback_expert; float my_val = 0.0f; bool my_bad = false;
+        for (int q = 0; q < EPL; ++q)
+            if (code[q] > lbest) { lbest = code[q]; lq = q; }
+    }
+    int my_id = fallback_expert; bool my_bad = false;
     for (int j = 0; j < p.k; ++j) {
-        const uint32_t wmax = __reduce_max_sync(full, lbest);
-        const unsigned ball = __ballot_sync(full, lbest == wmax);
-        const int src = __ffs(ball) - 1;                 // lowest lane = lowest expert id
-        const int sel_e = __shfl_sync(full, e0 + lq, src);
-        const float sel_v = __shfl_sync(full, lval, src);
-        const bool bad = wmax <= kCodeNegInf;            // nothing selectable is left
-        if (lane == j) {
-            my_id = bad ? fallback_expert : sel_e;
-            my_val = sel_v;
-            my_bad = bad;
-        }
-        if (lane == src && !bad) {
+        uint32_t m = lbest;
+#pragma unroll
+        for (int off = LPT / 2; off > 0; off >>= 1) m = max(m, __shfl_xor_sync(full, m, off, LPT));
+        const unsigned ball = __ballot_sync(full, lbest == m);
+        const unsigned seg = (ball >> (sub * LPT)) & ((LPT == 32) ? 0xffffffffu : ((1u << LPT) - 1u));
+        const int src = __ffs(seg) - 1;                  // lowest lane = lowest expert id
+        const int sel_e = __shfl_sync(full, e0 + lq, src, LPT);
+        const bool bad = m <= kCodeNegInf;               // nothing selectable is left
+        if (sl == j) { my_id = bad ? fallback_expert : sel_e; my_bad = bad; }
+        if (sl == src && !bad) {
 #pragma unroll
             for (int q = 0; q < EPL; ++q) if (q == lq) code[q] = 0;
-            lbest = 0; lq = 0; lval = 0.0f;
+            lbest = 0; lq = 0;
 #pragma unroll
             for (int q = 0; q < EPL; ++q)
-                if (code[q] > lbest) { lbest = code[q]; lq = q; lval = val[q]; }
+                if (code[q] > lbest) { lbest = code[q]; lq = q; }
         }
     }
 
-    // a5 weights: ratio of the chosen scores, summed and divided in double
+    // a5 weights: ratio of the chosen scores, summed and divided in double.  The score of a
+    // chosen expert is recomputed from its logit (same operations, same bits as above).
+    float my_val = 0.0f;
+    if (sl < p.k) {
+        const float lgv = __ldg(row + my_id);
+        my_val = sigmoid ? sigmoid_spec(lgv) : lgv;
+    }
+    const float v0 = __shfl_sync(full, my_val, 0, LPT);
     double u = 0.0;
-    const float v0 = __shfl_sync(full, my_val, 0);
-    if (lane < p.k) {
+    if (sl < p.k) {
         if (my_bad) u = 1.0;
-        else if (p.score_func == 0) u = exp((double)__fsub_rn(my_val, v0));
+        else if (!sigmoid) u = exp((double)__fsub_rn(my_val, v0));
         else u = (double)my_val;
     }
     double usum = 0.0;
-    for (int j = 0; j < p.k; ++j) usum += __shfl_sync(full, u, j);
+    for (int j = 0; j < p.k; ++j) usum += __shfl_sync(full, u, j, LPT);
     out_w = (float)((double)p.route_scale * u / usum);
 
     // a6 replica pick: (t mod live count)-th entry of the ascending live list
     out_id = my_id;
     out_slot = -1;
-    if (lane < p.k) {
+    if (sl < p.k) {
         const int n = s_nlive[my_id];
         out_slot = s_live[my_id * p.max_rep + (t % n)];
     }
     if (__any_sync(full, my_bad) && lane == 0) report_status(p.ctl, kDevInsufficientExperts);
 }
 
-template <int EPL>
-__global__ void __launch_bounds__(kRouteThreads) k_route(RouteParams p)
+template <int EPL, int LPT>
+__global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
 {
     extern __shared__ int32_t smem[];
     const int E = p.E, P = p.P, k = p.k, tb = p.tokens_per_block;
@@ -198,7 +198,7 @@ __global__ void __launch_bounds__(kRouteThreads) k_route(RouteParams p)
     int32_t *s_lrank = s_slot + NA;                   // [NA] stable rank inside the tile
     int32_t *s_hist = s_lrank + NA;                   // [P]  tile histogram (running)
     int32_t *s_excl = s_hist + P;                     // [P]  assignments on slot p in earlier tiles
-    int32_t *s_wcount = s_excl + P;                   // [8][P] per-warp counts of one round
+    uint16_t *s_wcount = reinterpret_cast<uint16_t *>(s_excl + P);   // [32][P] one round's counts
     __shared__ unsigned s_ticket, s_epoch;
     __shared__ int s_warp_sums[kRouteWarps];
 
@@ -223,7 +223,7 @@ __global__ void __launch_bounds__(kRouteThreads) k_route(RouteParams p)
         }
         s_nlive[e] = n;
     }
-    for (int q = tid; q < P; q += kRouteThreads) s_hist[q] = 0;
+    for (int q = tid; q < P; q += kRouteThreads) { s_hist[q] = 0; s_excl[q] = 0; }
     for (int q = tid; q < kRouteWarps * P; q += kRouteThreads) s_wcount[q] = 0;
     const int fallback_expert = p.state[0];
     __syncthreads();
@@ -233,83 +233,106 @@ __global__ void __launch_bounds__(kRouteThreads) k_route(RouteParams p)
     const int t0 = (int)ticket * tb;
     const int n_tok = min(tb, p.T - t0);
 
+    // which of this lane's experts have a live replica: the same for every token it routes
+    constexpr int kTokPerWarp = 32 / LPT;
+    const int sub = lane / LPT, sl = lane % LPT;
+    uint32_t avail_mask = 0;
+#pragma unroll
+    for (int q = 0; q < EPL; ++q) {
+        const int e = sl * EPL + q;
+        if (e < E && s_nlive[e] > 0) avail_mask |= 1u << q;
+    }
+
     // ---- a1..a6 per token -------------------------------------------------
-    for (int lt = warp; lt < tb; lt += kRouteWarps) {
+    for (int lt0 = warp * kTokPerWarp; lt0 < tb; lt0 += kRouteWarps * kTokPerWarp) {
+        const int lt = lt0 + sub;
         const int t = t0 + lt;
         int id = 0, slot = -1; float w = 0.0f;
-        if (t < p.T) {
-            route_token<EPL>(p, t, s_nlive, s_live, fallback_expert, id, w, slot);
-            if (lane < k) {
-                const size_t i = (size_t)t * k + lane;
+        if (t0 + lt0 < p.T) {                            // warp-uniform: some token of the warp exists
+            route_tokens<EPL, LPT>(p, t0 + lt0, avail_mask, s_nlive, s_live, fallback_expert, id, w, slot);
+            if (t >= p.T) slot = -1;
+            if (sl < k && t < p.T) {
+                const size_t i = (size_t)t * k + sl;
                 p.topk_ids[i] = id;
                 p.topk_weights[i] = w;
                 p.topk_slot[i] = slot;
             }
         }
-        if (lane < k) s_slot[lt * k + lane] = slot;
+        if (sl < k && lt < tb) s_slot[lt * k + sl] = slot;
     }
     __syncthreads();
 
     // ---- a7/a9 tile histogram and stable rank inside the tile --------------
-    // Rounds of 256 assignments in ascending i; inside a round, match_any gives
-    // the rank among equal slots of a warp and per-warp counts order the warps.
+    // Rounds of 1024 assignments in ascending i.  Inside a round, match_any gives
+    // the rank among equal slots of a warp and the per-warp counts; a scan down
+    // each slot's column of counts orders the warps.
     for (int base = 0; base < NA; base += kRouteThreads) {
         const int i = base + tid;
         const int slot = (i < NA) ? s_slot[i] : -1;
         const unsigned peers = __match_any_sync(full, slot);
         const int rank_in_warp = __popc(peers & lanemask_lt());
-        if (slot >= 0 && rank_in_warp == 0) s_wcount[warp * P + slot] = __popc(peers);
-        __syncthreads();
-        if (slot >= 0) {
-            int r = s_hist[slot] + rank_in_warp;
-            for (int w2 = 0; w2 < warp; ++w2) r += s_wcount[w2 * P + slot];
-            s_lrank[i] = r;
-        }
+        if (slot >= 0 && rank_in_warp == 0) s_wcount[warp * P + slot] = (uint16_t)__popc(peers);
         __syncthreads();
         for (int q = tid; q < P; q += kRouteThreads) {
-            int tot = 0;
-#pragma unroll
+            int run = s_hist[q];
+#pragma unroll 8
             for (int w2 = 0; w2 < kRouteWarps; ++w2) {
-                tot += s_wcount[w2 * P + q];
-                s_wcount[w2 * P + q] = 0;
+                const int c = s_wcount[w2 * P + q];
+                s_wcount[w2 * P + q] = (uint16_t)run;      // run < 65536: a tile has <= 32768 assignments
+                run += c;
             }
-            s_hist[q] += tot;
+            s_hist[q] = run;
         }
         __syncthreads();
+        if (slot >= 0) s_lrank[i] = (int)s_wcount[warp * P + slot] + rank_in_warp;
+        if (base + kRouteThreads < NA) {
+            __syncthreads();
+            for (int q = tid; q < kRouteWarps * P; q += kRouteThreads) s_wcount[q] = 0;
+            __syncthreads();
+        }
     }
 
-    // ---- a8 decoupled look-back over tiles, one thread per slot ------------
-    const bool last_tile = (ticket == gridDim.x - 1);
-    for (int q = tid; q < P; q += kRouteThreads) {
-        const unsigned long long mine = (unsigned long long)(unsigned)s_hist[q];
-        unsigned long long *d = p.desc + (size_t)ticket * P + q;
-        unsigned long long excl = 0;
-        if (ticket == 0) {
-            st_relaxed_u64(d, (epoch << 32) | (kFlagInclusive << 30) | mine);
-        } else {
-            st_relaxed_u64(d, (epoch << 32) | (kFlagAggregate << 30) | mine);
-            int b = (int)ticket - 1;
-            unsigned spins = 0;
-            bool gave_up = false;
-            while (true) {
-                const unsigned long long v = ld_relaxed_u64(p.desc + (size_t)b * P + q);
-                if ((v >> 32) != epoch) {                       // predecessor not there yet
-                    if (++spins > kSpinLimit ||
-                        ((spins & 1023u) == 0 && ld_relaxed_s32(&p.ctl->status) == kDevTimeout)) {
-                        gave_up = true;
-                        break;
-                    }
-                    __nanosleep(kSpinSleepNs);
-                    continue;
+    // ---- a8 prefix over tiles: publish this tile's aggregate, sum all earlier ones
+    for (int q = tid; q < P; q += kRouteThreads)
+        st_relaxed_u64(p.desc + (size_t)ticket * P + q, (epoch << 32) | (unsigned)s_hist[q]);
+    if (ticket > 0) {
+        // thread = (segment g, slot q): segment g sums tiles g, g+nseg, ... of column q,
+        // eight independent loads at a time
+        constexpr int kBatch = 8;
+        const int nseg = max(1, min(32, kRouteThreads / P));
+        const int per_pass = max(1, kRouteThreads / nseg);        // slots handled per pass
+        bool gave_up = false;
+        for (int q0 = 0; q0 < P; q0 += per_pass) {
+            const int g = tid / per_pass, q = q0 + tid % per_pass;
+            if (g >= nseg || q >= P) continue;
+            int partial = 0;
+            for (int b0 = g; b0 < (int)ticket && !gave_up; b0 += nseg * kBatch) {
+                unsigned long long v[kBatch];
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u) {
+                    const int b = b0 + u * nseg;
+                    v[u] = (b < (int)ticket) ? ld_relaxed_u64(p.desc + (size_t)b * P + q) : (epoch << 32);
                 }
-                excl += v & 0x3FFFFFFFull;
-                if (((v >> 30) & 3ull) == kFlagInclusive || b == 0) break;
-                --b;
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u) {
+                    const int b = b0 + u * nseg;
+                    unsigned spins = 0;
+                    while ((v[u] >> 32) != epoch) {                // that tile has not published yet
+                        if (++spins > kSpinLimit ||
+                            ((spins & 1023u) == 0 && ld_relaxed_s32(&p.ctl->status) == kDevTimeout)) {
+                            gave_up = true;
+                            break;
+                        }
+                        __nanosleep(kSpinSleepNs);
+                        v[u] = ld_relaxed_u64(p.desc + (size_t)b * P + q);
+                    }
+                    if (gave_up) break;
+                    partial += (int)(unsigned)(v[u] & 0xFFFFFFFFull);
+                }
             }
-            if (gave_up) report_status(p.ctl, kDevTimeout);
-            st_relaxed_u64(d, (epoch << 32) | (kFlagInclusive << 30) | ((excl + mine) & 0x3FFFFFFFull));
+            if (partial) atomicAdd(&s_excl[q], partial);
         }
-        s_excl[q] = (int)excl;
+        if (gave_up) report_status(p.ctl, kDevTimeout);
     }
     __syncthreads();
 
@@ -317,7 +340,7 @@ __global__ void __launch_bounds__(kRouteThreads) k_route(RouteParams p)
     for (int i = tid; i < n_tok * k; i += kRouteThreads)
         p.pos_in_slot[(size_t)t0 * k + i] = s_excl[s_slot[i]] + s_lrank[i];
 
-    if (!last_tile) return;
+    if (ticket != gridDim.x - 1) return;
 
     // ---- the last tile knows every total: a7 counts, a8 offsets -----------
     // exclusive scan over P with a contiguous chunk per thread
@@ -335,11 +358,10 @@ __global__ void __launch_bounds__(kRouteThreads) k_route(RouteParams p)
         if (lane >= off) incl += o;
     }
     if (lane == 31) s_warp_sums[warp] = incl;
-    __syncthreads();
+    __syncthreads();                                   // also: all reads of s_excl above are done
     int warp_base = 0;
     for (int w2 = 0; w2 < warp; ++w2) warp_base += s_warp_sums[w2];
     int run = warp_base + incl - local;
-    __syncthreads();                                   // s_excl is about to be overwritten
     for (int q = q0; q < min(P, q0 + chunk); ++q) {
         const int tot = s_hist[q];
         p.slot_counts[q] = tot;

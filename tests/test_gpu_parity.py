@@ -164,6 +164,23 @@ def test_bulk_copy_scatter_matches_oracle():
         os.environ.pop("MOE_BULK_STAGES", None)
 
 
+def test_combine_variants_match_oracle():
+    # the register (vector-load) combine and other shapes of the bulk-copy ring
+    settings = [{"MOE_COMBINE_IMPL": "0"},
+                {"MOE_COMBINE_IMPL": "1", "MOE_COMBINE_U": "2", "MOE_COMBINE_STAGES": "2"},
+                {"MOE_COMBINE_IMPL": "1", "MOE_COMBINE_U": "2", "MOE_COMBINE_STAGES": "6"},
+                {"MOE_COMBINE_IMPL": "1", "MOE_COMBINE_U": "4", "MOE_COMBINE_STAGES": "2"}]
+    for env in settings:
+        os.environ.update(env)
+        try:
+            for name, T, H in (("dsv3", 1037, None), ("mixtral", 300, 1000), ("tiny", 128, None), ("qwen3", 5, 8)):
+                wl = W.WORKLOADS[name]
+                run_and_check(wl, W.make_inputs(wl, T=T, H=H), wl.failure_sets[-1])
+        finally:
+            for key in env:
+                os.environ.pop(key, None)
+
+
 def test_step_from_host_memory():
     wl = W.WORKLOADS["dsv3"]
     T = 500
