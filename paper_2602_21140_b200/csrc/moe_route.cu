@@ -420,10 +420,10 @@ moe_status moe_route_init(const moe_config *cfg, const int32_t *slot_to_expert, 
         ctx->scatter_blocks_per_sm = std::max(1, env_int("MOE_SCATTER_BLOCKS_PER_SM", 8));
         ctx->combine_blocks_per_sm = std::max(1, env_int("MOE_COMBINE_BLOCKS_PER_SM", 8));
         ctx->combine_impl = env_int("MOE_COMBINE_IMPL", 1);
-        ctx->combine_u = env_int("MOE_COMBINE_U", 2);
+        ctx->combine_u = env_int("MOE_COMBINE_U", 1);
         if (ctx->combine_u != 1 && ctx->combine_u != 2 && ctx->combine_u != 4) ctx->combine_u = 2;
-        ctx->combine_warps = std::min(kCombineBulkMaxWarps, std::max(1, env_int("MOE_COMBINE_WARPS", 4)));
-        ctx->combine_stages = std::min(8, std::max(2, env_int("MOE_COMBINE_STAGES", 2)));
+        ctx->combine_warps = std::min(kCombineBulkMaxWarps, std::max(1, env_int("MOE_COMBINE_WARPS", 8)));
+        ctx->combine_stages = std::min(8, std::max(2, env_int("MOE_COMBINE_STAGES", 3)));
         while (ctx->combine_stages > 2 &&
                combine_bulk_smem(ctx->combine_stages, d.k, ctx->combine_u, ctx->combine_warps) > kMaxSmem - 1024)
             --ctx->combine_stages;
