@@ -367,7 +367,8 @@ def run_ours(args):
     dom = max(("k_scatter", "k_combine"), key=lambda n: dur_ms[n])
     achieved = alg[dom] / (dur_ms[dom] * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_source": f"of {peak_kind}", "traffic": NCU_TRAFFIC_BYTES[dom],
+                "frac": achieved / peak, "peak_source": f"of {peak_kind}",
+                "traffic": NCU_TRAFFIC_BYTES[dom] if (wl.name == "dsv3" and T == wl.T) else None,
                 "algorithmic_bytes": alg[dom], "kernel_ms": dur_ms[dom],
                 "per_kernel": {n: {"ms": dur_ms[n], "algorithmic_bytes": alg[n],
                                    "GB/s": alg[n] / (dur_ms[n] * 1e-3) / 1e9,
