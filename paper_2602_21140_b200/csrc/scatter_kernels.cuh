@@ -26,8 +26,6 @@ struct ScatterParams {
 };
 
 constexpr int kScatterThreads = 256;
-constexpr int kScatterUnroll = 4;                       // 16-byte loads in flight per lane
-constexpr int kScatterChunk = 32 * kScatterUnroll;      // uint4 per work item (2 KB)
 
 // a9 (final step): row = slot_offsets[slot] + rank inside the slot.  Lane j < k
 // owns assignment t*k + j.  Only read-only inputs are used, so any number of
@@ -47,29 +45,32 @@ __device__ __forceinline__ int resolve_row(const ScatterParams &p, int t, int la
     return row;
 }
 
+// UNROLL = 16-byte loads in flight per lane; a work item is 32*UNROLL 16-byte units of a row.
+template <int UNROLL>
 __global__ void __launch_bounds__(kScatterThreads) k_scatter_vec(ScatterParams p)
 {
+    constexpr int kChunk = 32 * UNROLL;
     const unsigned full = 0xffffffffu;
     const int lane = lane_id();
-    const int chunks = (p.hv + kScatterChunk - 1) / kScatterChunk;
+    const int chunks = (p.hv + kChunk - 1) / kChunk;
     const long long items = (long long)p.T * chunks;
     const long long warp0 = (long long)blockIdx.x * (kScatterThreads / 32) + (threadIdx.x >> 5);
     const long long nwarps = (long long)gridDim.x * (kScatterThreads / 32);
 
     for (long long it = warp0; it < items; it += nwarps) {
         const int t = (int)(it / chunks);
-        const int c0 = (int)(it % chunks) * kScatterChunk + lane;
+        const int c0 = (int)(it % chunks) * kChunk + lane;
         const uint4 *src = p.x + (size_t)t * p.hv;
-        uint4 v[kScatterUnroll];
+        uint4 v[UNROLL];
 #pragma unroll
-        for (int u = 0; u < kScatterUnroll; ++u)
+        for (int u = 0; u < UNROLL; ++u)
             if (c0 + 32 * u < p.hv) v[u] = ld_stream_v4(src + c0 + 32 * u);
         const int row = resolve_row(p, t, lane, it % chunks == 0);
         for (int j = 0; j < p.k; ++j) {
             const int r = __shfl_sync(full, row, j);
             uint4 *dst = p.send + (size_t)r * p.hv;
 #pragma unroll
-            for (int u = 0; u < kScatterUnroll; ++u)
+            for (int u = 0; u < UNROLL; ++u)
                 if (c0 + 32 * u < p.hv) st_stream_v4(dst + c0 + 32 * u, v[u]);
         }
     }
