@@ -132,6 +132,17 @@ moe_status moe_set_failed_ranks(moe_ctx *ctx, const int32_t *ranks, int32_t n, v
 moe_status moe_update_replica_map(moe_ctx *ctx, const int32_t *slot_to_expert, void *cuda_stream);
 
 /*
+ * moe_set_failed_experts — mark logical experts as lost one by one (Sec. 4.2:
+ * "selectively failing a fraction of the experts", their routing logits masked
+ * to minus infinity right before top-k), on top of whatever the failed-rank set
+ * already removes.  `mask` host [num_experts] u8, non-zero = lost; n must be
+ * num_experts, or 0 to clear the mask.  ABSOLUTE like moe_set_failed_ranks,
+ * same validation (INSUFFICIENT_EXPERTS if some token could be left with fewer
+ * than k experts), ordering and capture rules.
+ */
+moe_status moe_set_failed_experts(moe_ctx *ctx, const uint8_t *mask, int32_t n, void *cuda_stream);
+
+/*
  * moe_dispatch — gate, mask, select, count, scan, permute and scatter
  * (Sec. 2.1 gating and top-k; Sec. 2.3 dispatch / attention2expert).
  *   logits device [T,E] f32 row-major (finite; -inf acts as a mask)

@@ -147,10 +147,13 @@ uint16_t oracle_double_to_bf16(double d)
  * live[e*P .. e*P + n_live[e]) = slots p, ascending, with
  * slot_to_expert[p] == e whose rank p / S is not failed.  An expert is
  * available iff n_live[e] > 0: "Redundant experts" removes failed replicas
- * from the map, "Missing experts" masks an expert with none left.
+ * from the map, "Missing experts" masks an expert with none left.  An expert
+ * flagged in expert_failed (may be NULL) is lost whatever its replicas: the
+ * accuracy experiment of Sec. 4.2 fails experts one by one this way.
  */
 static void derive_live(const oracle_cfg *c, const int32_t *slot_to_expert,
-                        const uint8_t *rank_failed, int32_t *live, int32_t *n_live)
+                        const uint8_t *rank_failed, const uint8_t *expert_failed,
+                        int32_t *live, int32_t *n_live)
 {
     const int P = c->num_ranks * c->slots_per_rank;
     for (int e = 0; e < c->num_experts; ++e) n_live[e] = 0;
@@ -158,6 +161,7 @@ static void derive_live(const oracle_cfg *c, const int32_t *slot_to_expert,
         int e = slot_to_expert[p];
         if (e < 0) continue;                        /* empty slot */
         if (rank_failed[p / c->slots_per_rank]) continue;
+        if (expert_failed && expert_failed[e]) continue;    /* expert lost on its own (Sec. 4.2) */
         live[(size_t)e * P + n_live[e]++] = p;
     }
 }
@@ -171,12 +175,12 @@ static void derive_live(const oracle_cfg *c, const int32_t *slot_to_expert,
  * the fewest available experts (all non-empty groups if there are fewer).
  */
 int32_t oracle_failure_set_ok(const oracle_cfg *c, const int32_t *slot_to_expert,
-                              const uint8_t *rank_failed)
+                              const uint8_t *rank_failed, const uint8_t *expert_failed)
 {
     const int E = c->num_experts, P = c->num_ranks * c->slots_per_rank;
     int32_t *live = malloc((size_t)E * P * sizeof(int32_t));
     int32_t *n_live = malloc((size_t)E * sizeof(int32_t));
-    derive_live(c, slot_to_expert, rank_failed, live, n_live);
+    derive_live(c, slot_to_expert, rank_failed, expert_failed, live, n_live);
     int ok;
     if (c->n_group <= 1) {
         int avail = 0;
@@ -231,7 +235,7 @@ int32_t oracle_failure_set_ok(const oracle_cfg *c, const int32_t *slot_to_expert
  * Returns 0, or -1 if some token finds fewer than k finite keys.
  */
 int32_t oracle_route(const oracle_cfg *c, const int32_t *slot_to_expert,
-                     const uint8_t *rank_failed, const float *bias,
+                     const uint8_t *rank_failed, const uint8_t *expert_failed, const float *bias,
                      const float *logits, int32_t T,
                      int32_t *topk_ids, float *topk_weights, int32_t *topk_slot)
 {
@@ -243,7 +247,7 @@ int32_t oracle_route(const oracle_cfg *c, const int32_t *slot_to_expert,
     float *key = malloc((size_t)E * sizeof(float));
     uint8_t *picked = malloc((size_t)E);
     int rc = 0;
-    derive_live(c, slot_to_expert, rank_failed, live, n_live);
+    derive_live(c, slot_to_expert, rank_failed, expert_failed, live, n_live);
 
     for (int t = 0; t < T && rc == 0; ++t) {
         const float *lg = logits + (size_t)t * E;

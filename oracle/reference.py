@@ -118,16 +118,26 @@ def double_to_bf16(d) -> np.ndarray:
                     dtype=np.uint16).reshape(d.shape)
 
 
-def failure_set_ok(cfg: OracleConfig, slot_to_expert, failed_ranks) -> bool:
+def _expert_mask(cfg: OracleConfig, failed_experts):
+    if failed_experts is None:
+        return None
+    m = np.ascontiguousarray(np.asarray(failed_experts) != 0, dtype=np.uint8)
+    assert m.size == cfg.num_experts
+    return m
+
+
+def failure_set_ok(cfg: OracleConfig, slot_to_expert, failed_ranks, failed_experts=None) -> bool:
     lib = _load()
     s2e = _arr(slot_to_expert, np.int32)
     assert s2e.size == cfg.num_slots
     failed = _failed_mask(cfg, failed_ranks)
+    lost = _expert_mask(cfg, failed_experts)
     c = cfg._c()
-    return bool(lib.oracle_failure_set_ok(ctypes.byref(c), _p(s2e), _p(failed)))
+    return bool(lib.oracle_failure_set_ok(ctypes.byref(c), _p(s2e), _p(failed),
+                                          None if lost is None else _p(lost)))
 
 
-def route(cfg: OracleConfig, slot_to_expert, failed_ranks, bias, logits):
+def route(cfg: OracleConfig, slot_to_expert, failed_ranks, bias, logits, failed_experts=None):
     """Returns (topk_ids [T,k] i32, topk_weights [T,k] f32, topk_slot [T,k] i32)."""
     lib = _load()
     s2e = _arr(slot_to_expert, np.int32)
@@ -141,8 +151,9 @@ def route(cfg: OracleConfig, slot_to_expert, failed_ranks, bias, logits):
     ids = np.empty((T, k), np.int32)
     w = np.empty((T, k), np.float32)
     slot = np.empty((T, k), np.int32)
+    lost = _expert_mask(cfg, failed_experts)
     c = cfg._c()
-    rc = lib.oracle_route(ctypes.byref(c), _p(s2e), _p(failed),
+    rc = lib.oracle_route(ctypes.byref(c), _p(s2e), _p(failed), None if lost is None else _p(lost),
                           None if b is None else _p(b), _p(logits), ctypes.c_int32(T),
                           _p(ids), _p(w), _p(slot))
     if rc != 0:
@@ -195,9 +206,9 @@ def combine(buf_bf16, dst_row, topk_weights, topk_slot, slot_scale) -> np.ndarra
     return y
 
 
-def dispatch(cfg: OracleConfig, slot_to_expert, failed_ranks, bias, logits, x_bf16):
+def dispatch(cfg: OracleConfig, slot_to_expert, failed_ranks, bias, logits, x_bf16, failed_experts=None):
     """Route, count, permute and scatter: everything ``moe_dispatch`` produces."""
-    ids, w, slot = route(cfg, slot_to_expert, failed_ranks, bias, logits)
+    ids, w, slot = route(cfg, slot_to_expert, failed_ranks, bias, logits, failed_experts)
     out = permutation(cfg, slot)
     out.update(topk_ids=ids, topk_weights=w, topk_slot=slot)
     out["send_buf"] = scatter(x_bf16, out["dst_row"], cfg.top_k)

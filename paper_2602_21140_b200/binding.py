@@ -38,6 +38,7 @@ EXPORTED_SYMBOLS = (
     "moe_route_init", "moe_set_failed_ranks", "moe_update_replica_map", "moe_dispatch",
     "moe_combine", "moe_step_host", "moe_set_timing_event", "moe_get_device_status", "moe_plan_routing_state",
     "moe_workspace_bytes", "moe_route_destroy", "moe_status_string", "moe_permute_static",
+    "moe_set_failed_experts",
 )
 
 
@@ -81,6 +82,8 @@ def _lib():
         lib.moe_route_init.argtypes = [ctypes.POINTER(moe_config), vp, vp, vp, vp, ctypes.POINTER(vp)]
         lib.moe_set_failed_ranks.restype = ctypes.c_int
         lib.moe_set_failed_ranks.argtypes = [vp, vp, i32, vp]
+        lib.moe_set_failed_experts.restype = ctypes.c_int
+        lib.moe_set_failed_experts.argtypes = [vp, vp, i32, vp]
         lib.moe_update_replica_map.restype = ctypes.c_int
         lib.moe_update_replica_map.argtypes = [vp, vp, vp]
         lib.moe_dispatch.restype = ctypes.c_int
@@ -164,6 +167,13 @@ def moe_set_failed_ranks(ctx, ranks, cuda_stream: int = 0) -> int:
     r = _i32(list(ranks))
     return _lib().moe_set_failed_ranks(ctx, _np_ptr(r) if r.size else None, r.size,
                                        ctypes.c_void_p(cuda_stream))
+
+
+def moe_set_failed_experts(ctx, mask, cuda_stream: int = 0) -> int:
+    """mask: iterable of num_experts flags (non-zero = lost), or None / empty to clear."""
+    m = np.zeros(0, np.uint8) if mask is None else np.ascontiguousarray(np.asarray(mask) != 0, dtype=np.uint8)
+    return _lib().moe_set_failed_experts(ctx, _np_ptr(m) if m.size else None, m.size,
+                                         ctypes.c_void_p(cuda_stream))
 
 
 def moe_update_replica_map(ctx, slot_to_expert, cuda_stream: int = 0) -> int:
@@ -291,6 +301,11 @@ class MoeRouter:
         st = moe_set_failed_ranks(self._ctx, ranks, self._stream())
         if st != MOE_OK:
             raise MoeError(st, "moe_set_failed_ranks")
+
+    def set_failed_experts(self, mask) -> None:
+        st = moe_set_failed_experts(self._ctx, mask, self._stream())
+        if st != MOE_OK:
+            raise MoeError(st, "moe_set_failed_experts")
 
     def update_replica_map(self, slot_to_expert) -> None:
         st = moe_update_replica_map(self._ctx, slot_to_expert, self._stream())

@@ -35,6 +35,7 @@ struct Derived {
     int lanes_per_group;   // lanes holding one expert group (power of two), 0 if ungrouped
     int group_m;           // keys summed into a group score
     int rank_words;        // words of the rank bitmap
+    int expert_words;      // words of the failed-expert bitmap
     int state_words;       // words of the whole routing-state blob
     int tokens_per_block;  // routing tile
 };
@@ -99,7 +100,8 @@ bool derive(const moe_config *c, Derived *d)
     }
     if (d->epl == 0) return false;
     d->rank_words = (d->R + 31) / 32;
-    d->state_words = kStateHeaderWords + d->rank_words + d->E * d->max_rep;
+    d->expert_words = (d->E + 31) / 32;
+    d->state_words = kStateHeaderWords + d->rank_words + d->expert_words + d->E * d->max_rep;
     // routing tile: a power of two, grown with max_tokens so that a step has <= 128 tiles
     d->tokens_per_block = 32;
     while ((c->max_tokens + d->tokens_per_block - 1) / d->tokens_per_block > kMaxRouteTiles)
@@ -115,15 +117,19 @@ bool derive(const moe_config *c, Derived *d)
 // find k experts.  `blob` receives the device layout documented in
 // route_kernels.cuh.
 moe_status plan_state(const moe_config *c, const Derived &d, const int32_t *slot_to_expert,
-                      const std::vector<uint8_t> &failed, std::vector<int32_t> *blob,
-                      int *n_available)
+                      const std::vector<uint8_t> &failed, const std::vector<uint8_t> &expert_failed,
+                      std::vector<int32_t> *blob, int *n_available)
 {
     std::vector<int32_t> out((size_t)d.state_words, -1);
     uint32_t *alive = reinterpret_cast<uint32_t *>(out.data() + kStateHeaderWords);
     for (int w = 0; w < d.rank_words; ++w) alive[w] = 0u;
     for (int r = 0; r < d.R; ++r)
         if (!failed[r]) alive[r >> 5] |= 1u << (r & 31);
-    int32_t *table = out.data() + kStateHeaderWords + d.rank_words;
+    uint32_t *lost = reinterpret_cast<uint32_t *>(out.data() + kStateHeaderWords + d.rank_words);
+    for (int w = 0; w < d.expert_words; ++w) lost[w] = 0u;
+    for (int e = 0; e < d.E; ++e)
+        if (expert_failed[e]) lost[e >> 5] |= 1u << (e & 31);
+    int32_t *table = out.data() + kStateHeaderWords + d.rank_words + d.expert_words;
     std::vector<int> n_rep((size_t)d.E, 0), n_live((size_t)d.E, 0);
     for (int p = 0; p < d.P; ++p) {               // ascending p keeps each row ascending
         const int e = slot_to_expert[p];
@@ -131,7 +137,7 @@ moe_status plan_state(const moe_config *c, const Derived &d, const int32_t *slot
         if (e >= d.E) return MOE_ERR_INVALID_ARG;
         if (n_rep[e] == d.max_rep) return MOE_ERR_CAPACITY;
         table[e * d.max_rep + n_rep[e]++] = p;
-        if (!failed[p / d.S]) ++n_live[e];
+        if (!failed[p / d.S] && !expert_failed[e]) ++n_live[e];
     }
     int avail = 0, fallback = -1;
     for (int e = 0; e < d.E; ++e)
@@ -171,6 +177,7 @@ struct moe_ctx {
     // host mirror of the routing state
     std::vector<int32_t> slot_to_expert;
     std::vector<uint8_t> failed;
+    std::vector<uint8_t> expert_failed;
     // device state
     int32_t *d_state;
     float *d_bias;
@@ -344,11 +351,12 @@ moe_status moe_plan_routing_state(const moe_config *cfg, const int32_t *slot_to_
     }
     std::vector<int32_t> blob;
     int avail = 0;
-    const moe_status st = plan_state(cfg, d, slot_to_expert, failed, &blob, &avail);
+    const std::vector<uint8_t> none((size_t)d.E, 0);
+    const moe_status st = plan_state(cfg, d, slot_to_expert, failed, none, &blob, &avail);
     if (st != MOE_OK) return st;
     if (rank_alive) std::memcpy(rank_alive, blob.data() + kStateHeaderWords, (size_t)d.rank_words * 4);
     if (replica_table)
-        std::memcpy(replica_table, blob.data() + kStateHeaderWords + d.rank_words,
+        std::memcpy(replica_table, blob.data() + kStateHeaderWords + d.rank_words + d.expert_words,
                     (size_t)d.E * d.max_rep * 4);
     if (n_available) *n_available = avail;
     return MOE_OK;
@@ -362,7 +370,8 @@ moe_status moe_route_init(const moe_config *cfg, const int32_t *slot_to_expert, 
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     std::vector<uint8_t> failed((size_t)d.R, 0);
     std::vector<int32_t> blob;
-    moe_status ms = plan_state(cfg, d, slot_to_expert, failed, &blob, nullptr);
+    const std::vector<uint8_t> no_lost((size_t)d.E, 0);
+    moe_status ms = plan_state(cfg, d, slot_to_expert, failed, no_lost, &blob, nullptr);
     if (ms != MOE_OK) return ms;
 
     moe_ctx *ctx = new (std::nothrow) moe_ctx();
@@ -370,6 +379,7 @@ moe_status moe_route_init(const moe_config *cfg, const int32_t *slot_to_expert, 
     ctx->cfg = *cfg; ctx->d = d;
     ctx->slot_to_expert.assign(slot_to_expert, slot_to_expert + d.P);
     ctx->failed = failed;
+    ctx->expert_failed = no_lost;
     ctx->last_weights = nullptr; ctx->last_slot = nullptr; ctx->last_dst_row = nullptr;
     ctx->last_T = -1;
     ctx->timing_event = nullptr;
@@ -475,11 +485,11 @@ moe_status moe_set_failed_ranks(moe_ctx *ctx, const int32_t *ranks, int32_t n, v
         failed[ranks[i]] = 1;
     }
     std::vector<int32_t> blob;
-    const moe_status ms = plan_state(&ctx->cfg, d, ctx->slot_to_expert.data(), failed, &blob, nullptr);
+    const moe_status ms = plan_state(&ctx->cfg, d, ctx->slot_to_expert.data(), failed, ctx->expert_failed, &blob, nullptr);
     if (ms != MOE_OK) return ms;
     if (stream_is_capturing(st)) return MOE_ERR_INVALID_ARG;
     // only the header and the rank bitmap change
-    const moe_status ps = push_state(ctx, blob, kStateHeaderWords + d.rank_words, st);
+    const moe_status ps = push_state(ctx, blob, kStateHeaderWords + d.rank_words + d.expert_words, st);
     if (ps == MOE_OK) ctx->failed.swap(failed);
     return ps;
 }
@@ -490,11 +500,27 @@ moe_status moe_update_replica_map(moe_ctx *ctx, const int32_t *slot_to_expert, v
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const Derived &d = ctx->d;
     std::vector<int32_t> blob;
-    const moe_status ms = plan_state(&ctx->cfg, d, slot_to_expert, ctx->failed, &blob, nullptr);
+    const moe_status ms = plan_state(&ctx->cfg, d, slot_to_expert, ctx->failed, ctx->expert_failed, &blob, nullptr);
     if (ms != MOE_OK) return ms;
     if (stream_is_capturing(st)) return MOE_ERR_INVALID_ARG;
     const moe_status ps = push_state(ctx, blob, d.state_words, st);
     if (ps == MOE_OK) ctx->slot_to_expert.assign(slot_to_expert, slot_to_expert + d.P);
+    return ps;
+}
+
+moe_status moe_set_failed_experts(moe_ctx *ctx, const uint8_t *mask, int32_t n, void *cuda_stream)
+{
+    if (!ctx || (n != 0 && n != ctx->d.E) || (n > 0 && !mask)) return MOE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const Derived &d = ctx->d;
+    std::vector<uint8_t> lost((size_t)d.E, 0);
+    for (int e = 0; e < n; ++e) lost[e] = mask[e] ? 1 : 0;
+    std::vector<int32_t> blob;
+    const moe_status ms = plan_state(&ctx->cfg, d, ctx->slot_to_expert.data(), ctx->failed, lost, &blob, nullptr);
+    if (ms != MOE_OK) return ms;
+    if (stream_is_capturing(st)) return MOE_ERR_INVALID_ARG;
+    const moe_status ps = push_state(ctx, blob, kStateHeaderWords + d.rank_words + d.expert_words, st);
+    if (ps == MOE_OK) ctx->expert_failed.swap(lost);
     return ps;
 }
 
@@ -525,6 +551,7 @@ moe_status moe_dispatch(moe_ctx *ctx, const float *logits, const void *x, int32_
     rp.topk_group = ctx->cfg.topk_group; rp.lanes_per_group = d.lanes_per_group;
     rp.group_m = d.group_m; rp.route_scale = ctx->cfg.route_scale;
     rp.tokens_per_block = d.tokens_per_block; rp.rank_words = d.rank_words;
+    rp.expert_words = d.expert_words;
     rp.state = ctx->d_state; rp.bias = ctx->d_bias;
     rp.topk_ids = out->topk_ids; rp.topk_weights = out->topk_weights; rp.topk_slot = out->topk_slot;
     rp.pos_in_slot = ctx->d_pos;

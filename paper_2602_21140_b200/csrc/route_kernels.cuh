@@ -29,7 +29,8 @@ constexpr int kRouteWarps = kRouteThreads / 32;
 // Routing state blob in device memory (int32 words), rewritten by a remap:
 //   [0] fallback expert (lowest available id)   [1] number of available experts
 //   [2 .. 2+rank_words)  rank-alive bitmap, bit r of word r/32 set = rank r alive
-//   [2+rank_words ...)   replica table [E][max_rep]: ascending slot ids, -1 padded
+//   [.. +expert_words)   failed-expert bitmap, bit e set = expert e masked whatever its replicas
+//   [...]                replica table [E][max_rep]: ascending slot ids, -1 padded
 constexpr int kStateHeaderWords = 2;
 
 // Look-back descriptor, one 64-bit word per (tile, slot):
@@ -42,7 +43,7 @@ struct RouteParams {
     int score_func, n_group, topk_group, lanes_per_group, group_m;
     float route_scale;
     int tokens_per_block;
-    int rank_words;
+    int rank_words, expert_words;
     const int32_t *state;     // routing state blob
     const float *bias;        // [E]
     int32_t *topk_ids;        // [T,k]
@@ -211,10 +212,12 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
     }
     // Live replica lists from the rank bitmap and the replica table (a2, a6).
     const uint32_t *alive = reinterpret_cast<const uint32_t *>(p.state + kStateHeaderWords);
-    const int32_t *table = p.state + kStateHeaderWords + p.rank_words;
+    const uint32_t *lost = alive + p.rank_words;
+    const int32_t *table = p.state + kStateHeaderWords + p.rank_words + p.expert_words;
     for (int e = tid; e < E; e += kRouteThreads) {
         int n = 0;
-        for (int r = 0; r < p.max_rep; ++r) {
+        const bool expert_ok = !((lost[e >> 5] >> (e & 31)) & 1u);
+        for (int r = 0; r < p.max_rep && expert_ok; ++r) {
             const int slot = table[e * p.max_rep + r];
             if (slot >= 0) {
                 const int rank = slot / p.S;

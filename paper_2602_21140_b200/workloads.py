@@ -156,3 +156,26 @@ def make_inputs(wl: Workload, T: int | None = None, H: int | None = None,
     out["slot_scale"] = _rng(seed, 4).uniform(0.5, 1.5, wl.P).astype(np.float32)
     out["slot_to_expert"] = slot_to_expert(wl)
     return out
+
+
+# --------------------------------------------------------------------------
+# Expert-level failure generators (the two selection policies of the paper's
+# lost-expert experiment, Sec. 4.2).  They only choose WHICH experts fail.
+# --------------------------------------------------------------------------
+
+def every_nth_mask(E: int, r: float) -> np.ndarray:
+    """Uniform policy: fail experts at a fixed step so that a fraction r is lost
+    (r = 1/2 fails every even-indexed expert)."""
+    step = int(round(1.0 / r))
+    return (np.arange(E) % step == 0).astype(np.uint8)
+
+
+def most_activated_mask(activation_counts, r: float) -> np.ndarray:
+    """Worst-case policy: fail the fraction r of experts that were activated most
+    often (counts aggregated by the caller; ties go to the lower expert id)."""
+    counts = np.asarray(activation_counts, dtype=np.int64)
+    n = int(round(r * counts.size))
+    order = np.argsort(-counts, kind="stable")
+    mask = np.zeros(counts.size, np.uint8)
+    mask[order[:n]] = 1
+    return mask
