@@ -143,6 +143,37 @@ moe_status moe_update_replica_map(moe_ctx *ctx, const int32_t *slot_to_expert, v
 moe_status moe_set_failed_experts(moe_ctx *ctx, const uint8_t *mask, int32_t n, void *cuda_stream);
 
 /*
+ * moe_compact_ranks — host only, no CUDA call: the logical-rank reassignment of
+ * Sec. 3.5.  When a device with logical rank l_A fails it leaves a gap; the
+ * device at l_A + 1 takes l_A and every later one moves down by one.  With a
+ * role switch, the switched device (`switched_rank`, alive) takes the logical
+ * rank of the failed device it replaces (`replaced_rank`, failed) and the gap
+ * it leaves behind is closed the same way; pass -1, -1 for no role switch.
+ * Ranks are numbered by their original logical rank 0..num_ranks-1.
+ * Writes the physical (original) rank at each new logical rank to
+ * logical_to_physical[0 .. *n_logical), which must have room for num_ranks.
+ */
+moe_status moe_compact_ranks(int32_t num_ranks, const int32_t *failed_ranks, int32_t n_failed,
+                             int32_t switched_rank, int32_t replaced_rank,
+                             int32_t *logical_to_physical, int32_t *n_logical);
+
+/*
+ * moe_set_rank_order — lay the send buffer out in logical-rank order (Sec. 3.5:
+ * the communication domain is rebuilt with compacted ranks).
+ * logical_to_physical host [n] lists distinct physical ranks; the send buffer
+ * then holds the rows of rank logical_to_physical[0] first, and so on.  Every
+ * rank that is not failed must be listed (INVALID_ARG otherwise, also from a
+ * later moe_set_failed_ranks that would revive an unlisted rank); unlisted
+ * ranks own no rows.  n = 0 restores the physical numbering.  After this call
+ * rank_counts[l] and rank_offsets[l] of moe_dispatch_out refer to the l-th
+ * rank of the order, slot_counts / slot_offsets stay indexed by physical slot
+ * (slot_offsets is then no longer monotone in the slot id).  Same ordering and
+ * capture rules as moe_set_failed_ranks.
+ */
+moe_status moe_set_rank_order(moe_ctx *ctx, const int32_t *logical_to_physical, int32_t n,
+                              void *cuda_stream);
+
+/*
  * moe_dispatch — gate, mask, select, count, scan, permute and scatter
  * (Sec. 2.1 gating and top-k; Sec. 2.3 dispatch / attention2expert).
  *   logits device [T,E] f32 row-major (finite; -inf acts as a mask)

@@ -8,6 +8,7 @@ from .reference import (  # noqa: F401
     OracleConfig,
     build,
     combine,
+    compact_ranks,
     dispatch,
     double_to_bf16,
     exp_spec,

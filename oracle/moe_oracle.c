@@ -334,16 +334,20 @@ int32_t oracle_route(const oracle_cfg *c, const int32_t *slot_to_expert,
 /* ------------------------------------------------------------------------ */
 
 /*
- * slot_counts[p] = number of assignments i (i = t*k + j) with slot_i == p;
- * slot_offsets = exclusive prefix sum, slot_offsets[P] = T*k;
- * rank_counts[r] = sum over the rank's slots; rank_offsets[r] =
- * slot_offsets[r*S], rank_offsets[R] = T*k.  Walking i upward,
+ * slot_counts[p] = number of assignments i (i = t*k + j) with slot_i == p.
+ * The send buffer lists the ranks in `rank_order` (physical rank at each logical
+ * position, a permutation of 0..R-1; NULL = identity): Sec. 3.5 rebuilds the
+ * communication domain with compacted logical ranks, so the layout follows the
+ * logical numbering.  Walking the slots in that order (rank by rank, the S
+ * slots of a rank ascending), slot_offsets[p] = rows before slot p, and
+ * slot_offsets[P] = T*k.  rank_counts[l] / rank_offsets[l] belong to the l-th
+ * rank of the order, rank_offsets[R] = T*k.  Walking i upward,
  * dst_row[i] = slot_offsets[p] + (assignments seen so far on p), so the rows
  * of one slot keep ascending i; src_index is the inverse permutation.
- * The send buffer is expert-contiguous and rank-major: rank r owns rows
- * [rank_offsets[r], rank_offsets[r+1]), a failed rank owns none.
+ * A failed rank receives no assignment, hence owns no rows.
  */
 void oracle_permutation(const oracle_cfg *c, const int32_t *topk_slot, int32_t T,
+                        const int32_t *rank_order,
                         int32_t *slot_counts, int32_t *slot_offsets,
                         int32_t *rank_counts, int32_t *rank_offsets,
                         int32_t *dst_row, int32_t *src_index)
@@ -352,14 +356,20 @@ void oracle_permutation(const oracle_cfg *c, const int32_t *topk_slot, int32_t T
     const int64_t n = (int64_t)T * c->top_k;
     for (int p = 0; p < P; ++p) slot_counts[p] = 0;
     for (int64_t i = 0; i < n; ++i) slot_counts[topk_slot[i]]++;
-    slot_offsets[0] = 0;
-    for (int p = 0; p < P; ++p) slot_offsets[p + 1] = slot_offsets[p] + slot_counts[p];
-    for (int r = 0; r < R; ++r) {
-        rank_counts[r] = 0;
-        for (int s = 0; s < S; ++s) rank_counts[r] += slot_counts[r * S + s];
-        rank_offsets[r] = slot_offsets[r * S];
+    int32_t run = 0;
+    for (int l = 0; l < R; ++l) {
+        const int r = rank_order ? rank_order[l] : l;
+        rank_offsets[l] = run;
+        rank_counts[l] = 0;
+        for (int s = 0; s < S; ++s) {
+            const int p = r * S + s;
+            slot_offsets[p] = run;
+            run += slot_counts[p];
+            rank_counts[l] += slot_counts[p];
+        }
     }
-    rank_offsets[R] = slot_offsets[P];
+    slot_offsets[P] = run;
+    rank_offsets[R] = run;
     int32_t *seen = calloc((size_t)P, sizeof(int32_t));
     for (int64_t i = 0; i < n; ++i) {
         int p = topk_slot[i];
@@ -367,6 +377,37 @@ void oracle_permutation(const oracle_cfg *c, const int32_t *topk_slot, int32_t T
         src_index[dst_row[i]] = (int32_t)i;
     }
     free(seen);
+}
+
+/*
+ * Logical-rank reassignment of Sec. 3.5.  Ranks are named by their original
+ * logical rank.  A failed rank leaves a gap and every later rank moves down by
+ * one; with a role switch the switched rank first takes the place of the failed
+ * rank it replaces, and the place it vacates closes like any other gap.
+ * Returns the number of logical ranks written to order[].
+ */
+int32_t oracle_compact_ranks(int32_t R, const uint8_t *rank_failed, int32_t switched_rank,
+                             int32_t replaced_rank, int32_t *order)
+{
+    int32_t *cur = malloc((size_t)R * sizeof(int32_t));
+    int n = R;
+    for (int r = 0; r < R; ++r) cur[r] = r;
+    if (switched_rank >= 0) {
+        for (int i = 0; i < n; ++i) if (cur[i] == replaced_rank) cur[i] = switched_rank;   /* C takes l_A */
+        int seen = 0;
+        for (int i = 0; i < n; ++i) {                    /* the position C left is a gap: close it */
+            if (cur[i] == switched_rank && i != replaced_rank) { seen = 1; continue; }
+            cur[i - seen] = cur[i];
+        }
+        n -= seen;
+    }
+    int m = 0;
+    for (int i = 0; i < n; ++i) {                        /* close the gaps of the (other) failed ranks */
+        if (cur[i] != switched_rank && rank_failed[cur[i]]) continue;
+        order[m++] = cur[i];
+    }
+    free(cur);
+    return m;
 }
 
 /* ------------------------------------------------------------------------ */

@@ -74,6 +74,7 @@ def _load():
         lib.oracle_failure_set_ok.restype = ctypes.c_int32
         lib.oracle_route.restype = ctypes.c_int32
         lib.oracle_permutation.restype = None
+        lib.oracle_compact_ranks.restype = ctypes.c_int32
         lib.oracle_scatter.restype = None
         lib.oracle_combine.restype = None
         _lib = lib
@@ -161,8 +162,29 @@ def route(cfg: OracleConfig, slot_to_expert, failed_ranks, bias, logits, failed_
     return ids, w, slot
 
 
-def permutation(cfg: OracleConfig, topk_slot):
+def full_rank_order(cfg: OracleConfig, rank_order):
+    """The listed ranks first, then the unlisted ones ascending (they own no rows)."""
+    if rank_order is None:
+        return None
+    listed = [int(r) for r in rank_order]
+    rest = [r for r in range(cfg.num_ranks) if r not in listed]
+    return _arr(listed + rest, np.int32)
+
+
+def compact_ranks(num_ranks: int, failed_ranks, switched_rank: int = -1, replaced_rank: int = -1):
     lib = _load()
+    failed = np.zeros(num_ranks, np.uint8)
+    for r in failed_ranks:
+        failed[int(r)] = 1
+    out = np.full(num_ranks, -1, np.int32)
+    n = lib.oracle_compact_ranks(ctypes.c_int32(num_ranks), _p(failed), ctypes.c_int32(switched_rank),
+                                 ctypes.c_int32(replaced_rank), _p(out))
+    return out[:n].tolist()
+
+
+def permutation(cfg: OracleConfig, topk_slot, rank_order=None):
+    lib = _load()
+    order = full_rank_order(cfg, rank_order)
     slot = _arr(topk_slot, np.int32)
     T, k = slot.shape
     assert k == cfg.top_k
@@ -172,6 +194,7 @@ def permutation(cfg: OracleConfig, topk_slot):
                dst_row=np.empty(T * k, np.int32), src_index=np.empty(T * k, np.int32))
     c = cfg._c()
     lib.oracle_permutation(ctypes.byref(c), _p(slot), ctypes.c_int32(T),
+                           None if order is None else _p(order),
                            _p(out["slot_counts"]), _p(out["slot_offsets"]),
                            _p(out["rank_counts"]), _p(out["rank_offsets"]),
                            _p(out["dst_row"]), _p(out["src_index"]))
@@ -206,10 +229,11 @@ def combine(buf_bf16, dst_row, topk_weights, topk_slot, slot_scale) -> np.ndarra
     return y
 
 
-def dispatch(cfg: OracleConfig, slot_to_expert, failed_ranks, bias, logits, x_bf16, failed_experts=None):
+def dispatch(cfg: OracleConfig, slot_to_expert, failed_ranks, bias, logits, x_bf16, failed_experts=None,
+             rank_order=None):
     """Route, count, permute and scatter: everything ``moe_dispatch`` produces."""
     ids, w, slot = route(cfg, slot_to_expert, failed_ranks, bias, logits, failed_experts)
-    out = permutation(cfg, slot)
+    out = permutation(cfg, slot, rank_order)
     out.update(topk_ids=ids, topk_weights=w, topk_slot=slot)
     out["send_buf"] = scatter(x_bf16, out["dst_row"], cfg.top_k)
     return out

@@ -38,7 +38,7 @@ EXPORTED_SYMBOLS = (
     "moe_route_init", "moe_set_failed_ranks", "moe_update_replica_map", "moe_dispatch",
     "moe_combine", "moe_step_host", "moe_set_timing_event", "moe_get_device_status", "moe_plan_routing_state",
     "moe_workspace_bytes", "moe_route_destroy", "moe_status_string", "moe_permute_static",
-    "moe_set_failed_experts",
+    "moe_set_failed_experts", "moe_compact_ranks", "moe_set_rank_order",
 )
 
 
@@ -84,6 +84,10 @@ def _lib():
         lib.moe_set_failed_ranks.argtypes = [vp, vp, i32, vp]
         lib.moe_set_failed_experts.restype = ctypes.c_int
         lib.moe_set_failed_experts.argtypes = [vp, vp, i32, vp]
+        lib.moe_compact_ranks.restype = ctypes.c_int
+        lib.moe_compact_ranks.argtypes = [i32, vp, i32, i32, i32, vp, ctypes.POINTER(i32)]
+        lib.moe_set_rank_order.restype = ctypes.c_int
+        lib.moe_set_rank_order.argtypes = [vp, vp, i32, vp]
         lib.moe_update_replica_map.restype = ctypes.c_int
         lib.moe_update_replica_map.argtypes = [vp, vp, vp]
         lib.moe_dispatch.restype = ctypes.c_int
@@ -174,6 +178,21 @@ def moe_set_failed_experts(ctx, mask, cuda_stream: int = 0) -> int:
     m = np.zeros(0, np.uint8) if mask is None else np.ascontiguousarray(np.asarray(mask) != 0, dtype=np.uint8)
     return _lib().moe_set_failed_experts(ctx, _np_ptr(m) if m.size else None, m.size,
                                          ctypes.c_void_p(cuda_stream))
+
+
+def moe_compact_ranks(num_ranks: int, failed_ranks, switched_rank: int = -1, replaced_rank: int = -1):
+    """Host-only rank compaction.  Returns (status, list of physical ranks in new logical order)."""
+    fr = _i32(list(failed_ranks))
+    out = np.full(max(num_ranks, 1), -1, np.int32)
+    n = ctypes.c_int32(0)
+    st = _lib().moe_compact_ranks(num_ranks, _np_ptr(fr) if fr.size else None, fr.size, switched_rank,
+                                  replaced_rank, _np_ptr(out), ctypes.byref(n))
+    return st, out[: n.value].tolist()
+
+
+def moe_set_rank_order(ctx, logical_to_physical, cuda_stream: int = 0) -> int:
+    o = _i32(list(logical_to_physical))
+    return _lib().moe_set_rank_order(ctx, _np_ptr(o) if o.size else None, o.size, ctypes.c_void_p(cuda_stream))
 
 
 def moe_update_replica_map(ctx, slot_to_expert, cuda_stream: int = 0) -> int:
@@ -306,6 +325,11 @@ class MoeRouter:
         st = moe_set_failed_experts(self._ctx, mask, self._stream())
         if st != MOE_OK:
             raise MoeError(st, "moe_set_failed_experts")
+
+    def set_rank_order(self, logical_to_physical) -> None:
+        st = moe_set_rank_order(self._ctx, logical_to_physical, self._stream())
+        if st != MOE_OK:
+            raise MoeError(st, "moe_set_rank_order")
 
     def update_replica_map(self, slot_to_expert) -> None:
         st = moe_update_replica_map(self._ctx, slot_to_expert, self._stream())

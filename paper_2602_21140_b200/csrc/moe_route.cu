@@ -101,7 +101,7 @@ bool derive(const moe_config *c, Derived *d)
     if (d->epl == 0) return false;
     d->rank_words = (d->R + 31) / 32;
     d->expert_words = (d->E + 31) / 32;
-    d->state_words = kStateHeaderWords + d->rank_words + d->expert_words + d->E * d->max_rep;
+    d->state_words = kStateHeaderWords + d->rank_words + d->expert_words + d->E * d->max_rep + d->P;
     // routing tile: a power of two, grown with max_tokens so that a step has <= 128 tiles
     d->tokens_per_block = 32;
     while ((c->max_tokens + d->tokens_per_block - 1) / d->tokens_per_block > kMaxRouteTiles)
@@ -118,8 +118,16 @@ bool derive(const moe_config *c, Derived *d)
 // route_kernels.cuh.
 moe_status plan_state(const moe_config *c, const Derived &d, const int32_t *slot_to_expert,
                       const std::vector<uint8_t> &failed, const std::vector<uint8_t> &expert_failed,
+                      const std::vector<int32_t> &rank_order, int n_listed,
                       std::vector<int32_t> *blob, int *n_available)
 {
+    // the layout order must give every alive rank a place among the listed ranks
+    {
+        std::vector<uint8_t> listed((size_t)d.R, 0);
+        for (int i = 0; i < n_listed; ++i) listed[rank_order[i]] = 1;
+        for (int r = 0; r < d.R; ++r)
+            if (!failed[r] && !listed[r]) return MOE_ERR_INVALID_ARG;
+    }
     std::vector<int32_t> out((size_t)d.state_words, -1);
     uint32_t *alive = reinterpret_cast<uint32_t *>(out.data() + kStateHeaderWords);
     for (int w = 0; w < d.rank_words; ++w) alive[w] = 0u;
@@ -160,6 +168,9 @@ moe_status plan_state(const moe_config *c, const Derived &d, const int32_t *slot
         ok = worst >= d.k;
     }
     if (!ok) return MOE_ERR_INSUFFICIENT_EXPERTS;
+    int32_t *order = table + d.E * d.max_rep;          // send-buffer layout: slots in logical-rank order
+    for (int l = 0; l < d.R; ++l)
+        for (int sl = 0; sl < d.S; ++sl) order[l * d.S + sl] = rank_order[l] * d.S + sl;
     out[0] = fallback;
     out[1] = avail;
     if (blob) blob->swap(out);
@@ -178,6 +189,8 @@ struct moe_ctx {
     std::vector<int32_t> slot_to_expert;
     std::vector<uint8_t> failed;
     std::vector<uint8_t> expert_failed;
+    std::vector<int32_t> rank_order;   // physical rank at each logical position (full permutation)
+    int n_listed;                      // leading entries given by the caller; the rest own no rows
     // device state
     int32_t *d_state;
     float *d_bias;
@@ -352,7 +365,9 @@ moe_status moe_plan_routing_state(const moe_config *cfg, const int32_t *slot_to_
     std::vector<int32_t> blob;
     int avail = 0;
     const std::vector<uint8_t> none((size_t)d.E, 0);
-    const moe_status st = plan_state(cfg, d, slot_to_expert, failed, none, &blob, &avail);
+    std::vector<int32_t> ident((size_t)d.R);
+    for (int r = 0; r < d.R; ++r) ident[r] = r;
+    const moe_status st = plan_state(cfg, d, slot_to_expert, failed, none, ident, d.R, &blob, &avail);
     if (st != MOE_OK) return st;
     if (rank_alive) std::memcpy(rank_alive, blob.data() + kStateHeaderWords, (size_t)d.rank_words * 4);
     if (replica_table)
@@ -371,7 +386,9 @@ moe_status moe_route_init(const moe_config *cfg, const int32_t *slot_to_expert, 
     std::vector<uint8_t> failed((size_t)d.R, 0);
     std::vector<int32_t> blob;
     const std::vector<uint8_t> no_lost((size_t)d.E, 0);
-    moe_status ms = plan_state(cfg, d, slot_to_expert, failed, no_lost, &blob, nullptr);
+    std::vector<int32_t> ident((size_t)d.R);
+    for (int r = 0; r < d.R; ++r) ident[r] = r;
+    moe_status ms = plan_state(cfg, d, slot_to_expert, failed, no_lost, ident, d.R, &blob, nullptr);
     if (ms != MOE_OK) return ms;
 
     moe_ctx *ctx = new (std::nothrow) moe_ctx();
@@ -380,6 +397,8 @@ moe_status moe_route_init(const moe_config *cfg, const int32_t *slot_to_expert, 
     ctx->slot_to_expert.assign(slot_to_expert, slot_to_expert + d.P);
     ctx->failed = failed;
     ctx->expert_failed = no_lost;
+    ctx->rank_order = ident;
+    ctx->n_listed = d.R;
     ctx->last_weights = nullptr; ctx->last_slot = nullptr; ctx->last_dst_row = nullptr;
     ctx->last_T = -1;
     ctx->timing_event = nullptr;
@@ -485,7 +504,8 @@ moe_status moe_set_failed_ranks(moe_ctx *ctx, const int32_t *ranks, int32_t n, v
         failed[ranks[i]] = 1;
     }
     std::vector<int32_t> blob;
-    const moe_status ms = plan_state(&ctx->cfg, d, ctx->slot_to_expert.data(), failed, ctx->expert_failed, &blob, nullptr);
+    const moe_status ms = plan_state(&ctx->cfg, d, ctx->slot_to_expert.data(), failed, ctx->expert_failed, ctx->rank_order,
+                                     ctx->n_listed, &blob, nullptr);
     if (ms != MOE_OK) return ms;
     if (stream_is_capturing(st)) return MOE_ERR_INVALID_ARG;
     // only the header and the rank bitmap change
@@ -500,7 +520,8 @@ moe_status moe_update_replica_map(moe_ctx *ctx, const int32_t *slot_to_expert, v
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const Derived &d = ctx->d;
     std::vector<int32_t> blob;
-    const moe_status ms = plan_state(&ctx->cfg, d, slot_to_expert, ctx->failed, ctx->expert_failed, &blob, nullptr);
+    const moe_status ms = plan_state(&ctx->cfg, d, slot_to_expert, ctx->failed, ctx->expert_failed, ctx->rank_order,
+                                     ctx->n_listed, &blob, nullptr);
     if (ms != MOE_OK) return ms;
     if (stream_is_capturing(st)) return MOE_ERR_INVALID_ARG;
     const moe_status ps = push_state(ctx, blob, d.state_words, st);
@@ -516,11 +537,72 @@ moe_status moe_set_failed_experts(moe_ctx *ctx, const uint8_t *mask, int32_t n, 
     std::vector<uint8_t> lost((size_t)d.E, 0);
     for (int e = 0; e < n; ++e) lost[e] = mask[e] ? 1 : 0;
     std::vector<int32_t> blob;
-    const moe_status ms = plan_state(&ctx->cfg, d, ctx->slot_to_expert.data(), ctx->failed, lost, &blob, nullptr);
+    const moe_status ms = plan_state(&ctx->cfg, d, ctx->slot_to_expert.data(), ctx->failed, lost, ctx->rank_order,
+                                     ctx->n_listed, &blob, nullptr);
     if (ms != MOE_OK) return ms;
     if (stream_is_capturing(st)) return MOE_ERR_INVALID_ARG;
     const moe_status ps = push_state(ctx, blob, kStateHeaderWords + d.rank_words + d.expert_words, st);
     if (ps == MOE_OK) ctx->expert_failed.swap(lost);
+    return ps;
+}
+
+moe_status moe_compact_ranks(int32_t num_ranks, const int32_t *failed_ranks, int32_t n_failed,
+                             int32_t switched_rank, int32_t replaced_rank,
+                             int32_t *logical_to_physical, int32_t *n_logical)
+{
+    if (num_ranks < 1 || n_failed < 0 || (n_failed > 0 && !failed_ranks) || !logical_to_physical || !n_logical)
+        return MOE_ERR_INVALID_ARG;
+    std::vector<uint8_t> failed((size_t)num_ranks, 0);
+    for (int i = 0; i < n_failed; ++i) {
+        if (failed_ranks[i] < 0 || failed_ranks[i] >= num_ranks) return MOE_ERR_INVALID_ARG;
+        failed[failed_ranks[i]] = 1;
+    }
+    const bool role_switch = switched_rank >= 0 || replaced_rank >= 0;
+    if (role_switch) {
+        if (switched_rank < 0 || switched_rank >= num_ranks || replaced_rank < 0 || replaced_rank >= num_ranks)
+            return MOE_ERR_INVALID_ARG;
+        if (failed[switched_rank] || !failed[replaced_rank]) return MOE_ERR_INVALID_ARG;
+    }
+    // walk the old logical order: the switched rank takes the failed rank's position, other
+    // failed ranks leave a gap that the following ranks close by moving down one
+    int n = 0;
+    for (int r = 0; r < num_ranks; ++r) {
+        if (role_switch && r == replaced_rank) { logical_to_physical[n++] = switched_rank; continue; }
+        if (role_switch && r == switched_rank) continue;
+        if (failed[r]) continue;
+        logical_to_physical[n++] = r;
+    }
+    *n_logical = n;
+    return MOE_OK;
+}
+
+moe_status moe_set_rank_order(moe_ctx *ctx, const int32_t *logical_to_physical, int32_t n, void *cuda_stream)
+{
+    if (!ctx || n < 0 || n > ctx->d.R || (n > 0 && !logical_to_physical)) return MOE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const Derived &d = ctx->d;
+    std::vector<int32_t> order;
+    std::vector<uint8_t> seen((size_t)d.R, 0);
+    if (n == 0) {                                        // back to the physical numbering
+        for (int r = 0; r < d.R; ++r) order.push_back(r);
+        n = d.R;
+    } else {
+        for (int i = 0; i < n; ++i) {
+            const int r = logical_to_physical[i];
+            if (r < 0 || r >= d.R || seen[r]) return MOE_ERR_INVALID_ARG;
+            seen[r] = 1;
+            order.push_back(r);
+        }
+        for (int r = 0; r < d.R; ++r)                    // unlisted ranks own no rows; keep a full permutation
+            if (!seen[r]) order.push_back(r);
+    }
+    std::vector<int32_t> blob;
+    const moe_status ms = plan_state(&ctx->cfg, d, ctx->slot_to_expert.data(), ctx->failed, ctx->expert_failed,
+                                     order, n, &blob, nullptr);
+    if (ms != MOE_OK) return ms;
+    if (stream_is_capturing(st)) return MOE_ERR_INVALID_ARG;
+    const moe_status ps = push_state(ctx, blob, d.state_words, st);
+    if (ps == MOE_OK) { ctx->rank_order.swap(order); ctx->n_listed = n; }
     return ps;
 }
 

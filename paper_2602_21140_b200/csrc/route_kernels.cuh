@@ -31,6 +31,8 @@ constexpr int kRouteWarps = kRouteThreads / 32;
 //   [2 .. 2+rank_words)  rank-alive bitmap, bit r of word r/32 set = rank r alive
 //   [.. +expert_words)   failed-expert bitmap, bit e set = expert e masked whatever its replicas
 //   [...]                replica table [E][max_rep]: ascending slot ids, -1 padded
+//   [...]                slot order [P]: physical slot at each position of the send-buffer
+//                        layout (logical-rank order; identity unless ranks were compacted)
 constexpr int kStateHeaderWords = 2;
 
 // Look-back descriptor, one 64-bit word per (tile, slot):
@@ -346,15 +348,15 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
     if (ticket != gridDim.x - 1) return;
 
     // ---- the last tile knows every total: a7 counts, a8 offsets -----------
-    // exclusive scan over P with a contiguous chunk per thread
+    // exclusive scan over the P layout positions (position q holds physical slot order[q]),
+    // a contiguous chunk of positions per thread
+    const int32_t *order = p.state + kStateHeaderWords + p.rank_words + p.expert_words + E * p.max_rep;
+    for (int q = tid; q < P; q += kRouteThreads) s_hist[q] += s_excl[q];     // totals per physical slot
+    __syncthreads();
     const int chunk = (P + kRouteThreads - 1) / kRouteThreads;
     const int q0 = tid * chunk;
     int local = 0;
-    for (int q = q0; q < min(P, q0 + chunk); ++q) {
-        const int tot = s_excl[q] + s_hist[q];
-        s_hist[q] = tot;
-        local += tot;
-    }
+    for (int q = q0; q < min(P, q0 + chunk); ++q) local += s_hist[order[q]];
     int incl = local;
     for (int off = 1; off < 32; off <<= 1) {
         const int o = __shfl_up_sync(full, incl, off);
@@ -366,10 +368,11 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
     for (int w2 = 0; w2 < warp; ++w2) warp_base += s_warp_sums[w2];
     int run = warp_base + incl - local;
     for (int q = q0; q < min(P, q0 + chunk); ++q) {
-        const int tot = s_hist[q];
-        p.slot_counts[q] = tot;
-        p.slot_offsets[q] = run;
-        s_excl[q] = run;
+        const int slot = order[q];
+        const int tot = s_hist[slot];
+        p.slot_counts[slot] = tot;
+        p.slot_offsets[slot] = run;
+        s_excl[q] = run;                               // offset of layout position q
         run += tot;
     }
     if (tid == kRouteThreads - 1) {
@@ -377,9 +380,9 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
         p.rank_offsets[p.R] = run;
     }
     __syncthreads();
-    for (int r = tid; r < p.R; r += kRouteThreads) {
+    for (int r = tid; r < p.R; r += kRouteThreads) {   // r-th rank of the layout order
         int c = 0;
-        for (int s = 0; s < p.S; ++s) c += s_hist[r * p.S + s];
+        for (int s = 0; s < p.S; ++s) c += s_hist[order[r * p.S + s]];
         p.rank_counts[r] = c;
         p.rank_offsets[r] = s_excl[r * p.S];
     }
