@@ -47,7 +47,14 @@ typedef enum {
     MOE_ERR_DEVICE_TIMEOUT = 5        /* a bounded device-side wait gave up (see get_device_status) */
 } moe_status;
 
-enum { MOE_SCORE_SOFTMAX = 0, MOE_SCORE_SIGMOID = 1 };
+/* score_func values.  MOE_ROUTE_DENSE_TP is the routing of the dense FFN layers of
+ * Sec. 3.4: num_experts = groups * top_k names the top_k tensor-parallel shards
+ * (expert g*top_k + s = shard s of FFN group g) of replicated FFN groups; a group
+ * with any shard lost is compromised and skipped, token t goes to all shards of
+ * the (t mod n_healthy)-th healthy group with weight route_scale, so tokens are
+ * spread evenly over the healthy groups.  Logits are not read in this mode (the
+ * pointer may be NULL); n_group must be 1 and groups <= 32 * top_k. */
+enum { MOE_SCORE_SOFTMAX = 0, MOE_SCORE_SIGMOID = 1, MOE_ROUTE_DENSE_TP = 2 };
 
 /* Limits of this build: num_experts <= 512, top_k <= 16, max_replicas <= 8,
  * num_ranks*slots_per_rank <= 4096, hidden % 8 == 0.  With n_group > 1:
@@ -61,7 +68,7 @@ typedef struct {
     int32_t num_ranks;      /* R: simulated EP ranks                                         */
     int32_t slots_per_rank; /* S: physical expert slots per rank                             */
     int32_t max_replicas;   /* most physical copies any logical expert may have              */
-    int32_t score_func;     /* MOE_SCORE_SOFTMAX | MOE_SCORE_SIGMOID (+ bias on the key)     */
+    int32_t score_func;     /* MOE_SCORE_SOFTMAX | MOE_SCORE_SIGMOID (+ bias on the key) | MOE_ROUTE_DENSE_TP */
     int32_t n_group;        /* 1 = plain top-k; > 1 = group-limited selection                */
     int32_t topk_group;     /* groups kept when n_group > 1                                  */
     int32_t replica_policy; /* 0 = replica (t mod live count) of the ascending live list     */

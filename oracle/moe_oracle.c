@@ -42,7 +42,7 @@ typedef struct {
     int32_t top_k;          /* k                                                   */
     int32_t num_ranks;      /* R  simulated EP ranks                               */
     int32_t slots_per_rank; /* S  physical slots per rank; slot p lives on p / S   */
-    int32_t score_func;     /* 0 softmax, 1 sigmoid (+ bias on the selection key)  */
+    int32_t score_func;     /* 0 softmax, 1 sigmoid (+ bias on the key), 2 dense TP groups */
     int32_t n_group;        /* 1 = no group-limited selection                      */
     int32_t topk_group;     /* groups kept when n_group > 1                        */
     float   route_scale;    /* multiplies the renormalised weights                 */
@@ -182,7 +182,14 @@ int32_t oracle_failure_set_ok(const oracle_cfg *c, const int32_t *slot_to_expert
     int32_t *n_live = malloc((size_t)E * sizeof(int32_t));
     derive_live(c, slot_to_expert, rank_failed, expert_failed, live, n_live);
     int ok;
-    if (c->n_group <= 1) {
+    if (c->score_func == 2) {                            /* dense: some group keeps all its shards */
+        ok = 0;
+        for (int g = 0; g < E / c->top_k; ++g) {
+            int all = 1;
+            for (int s = 0; s < c->top_k; ++s) all = all && n_live[g * c->top_k + s] > 0;
+            ok = ok || all;
+        }
+    } else if (c->n_group <= 1) {
         int avail = 0;
         for (int e = 0; e < E; ++e) avail += n_live[e] > 0;
         ok = avail >= c->top_k;
@@ -249,6 +256,33 @@ int32_t oracle_route(const oracle_cfg *c, const int32_t *slot_to_expert,
     int rc = 0;
     derive_live(c, slot_to_expert, rank_failed, expert_failed, live, n_live);
 
+    if (c->score_func == 2) {
+        /* Dense FFN layers (Sec. 3.4): the E "experts" are the k tensor-parallel shards of
+         * E/k replicated FFN groups.  A group that lost any shard is compromised; tokens are
+         * spread evenly over the healthy groups: token t goes to every shard of the
+         * (t mod n_healthy)-th healthy group, each with weight route_scale (the shards'
+         * partial results add up in combine). */
+        const int G = E / k;
+        int *healthy = malloc((size_t)G * sizeof(int));
+        int n_healthy = 0;
+        for (int g = 0; g < G; ++g) {
+            int all = 1;
+            for (int s = 0; s < k; ++s) all = all && n_live[g * k + s] > 0;
+            if (all) healthy[n_healthy++] = g;
+        }
+        if (n_healthy == 0) rc = -1;
+        for (int t = 0; t < T && rc == 0; ++t) {
+            const int g = healthy[t % n_healthy];
+            for (int j = 0; j < k; ++j) {
+                const int e = g * k + j;
+                topk_ids[(size_t)t * k + j] = e;
+                topk_weights[(size_t)t * k + j] = c->route_scale;
+                topk_slot[(size_t)t * k + j] = live[(size_t)e * P + (t % n_live[e])];
+            }
+        }
+        free(healthy);
+        T = 0;                                           /* nothing left for the gated path */
+    }
     for (int t = 0; t < T && rc == 0; ++t) {
         const float *lg = logits + (size_t)t * E;
         for (int e = 0; e < E; ++e) {

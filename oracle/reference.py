@@ -145,7 +145,7 @@ def route(cfg: OracleConfig, slot_to_expert, failed_ranks, bias, logits, failed_
     assert s2e.size == cfg.num_slots
     failed = _failed_mask(cfg, failed_ranks)
     logits = _arr(logits, np.float32)
-    T, E = logits.shape
+    T, E = logits.shape                       # dense mode (score_func 2) reads only the shape
     assert E == cfg.num_experts
     k = cfg.top_k
     b = None if bias is None else _arr(bias, np.float32)

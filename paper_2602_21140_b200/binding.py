@@ -33,6 +33,7 @@ MOE_ERR_CAPACITY = 4
 MOE_ERR_DEVICE_TIMEOUT = 5
 MOE_SCORE_SOFTMAX = 0
 MOE_SCORE_SIGMOID = 1
+MOE_ROUTE_DENSE_TP = 2
 
 EXPORTED_SYMBOLS = (
     "moe_route_init", "moe_set_failed_ranks", "moe_update_replica_map", "moe_dispatch",

@@ -59,7 +59,12 @@ bool derive(const moe_config *c, Derived *d)
     const long long P = (long long)c->num_ranks * c->slots_per_rank;
     if (P > kMaxSlots) return false;
     if (c->max_replicas < 1 || c->max_replicas > kMaxReplicas) return false;
-    if (c->score_func != MOE_SCORE_SOFTMAX && c->score_func != MOE_SCORE_SIGMOID) return false;
+    if (c->score_func != MOE_SCORE_SOFTMAX && c->score_func != MOE_SCORE_SIGMOID &&
+        c->score_func != MOE_ROUTE_DENSE_TP)
+        return false;
+    if (c->score_func == MOE_ROUTE_DENSE_TP &&
+        (c->n_group != 1 || c->num_experts % c->top_k != 0 || c->num_experts / c->top_k > 32 * c->top_k))
+        return false;
     if (c->replica_policy != 0) return false;
     if (!(c->route_scale > 0.0f)) return false;
     if ((long long)c->max_tokens * c->top_k >= (1ll << 30)) return false;   // 30-bit scan counts
@@ -151,7 +156,17 @@ moe_status plan_state(const moe_config *c, const Derived &d, const int32_t *slot
     for (int e = 0; e < d.E; ++e)
         if (n_live[e] > 0) { ++avail; if (fallback < 0) fallback = e; }
     bool ok;
-    if (c->n_group <= 1) {
+    if (c->score_func == MOE_ROUTE_DENSE_TP) {
+        // dense-FFN groups of k shards: at least one group must have every shard live
+        int healthy = 0;
+        for (int g = 0; g < d.E / d.k; ++g) {
+            bool all = true;
+            for (int sh = 0; sh < d.k; ++sh) all = all && n_live[g * d.k + sh] > 0;
+            healthy += all;
+        }
+        ok = healthy >= 1;
+        avail = healthy;
+    } else if (c->n_group <= 1) {
         ok = avail >= d.k;
     } else {
         // worst case: the kept groups are the non-empty ones with the fewest experts
@@ -620,7 +635,7 @@ moe_status moe_dispatch(moe_ctx *ctx, const float *logits, const void *x, int32_
         !out->slot_offsets || !out->rank_counts || !out->rank_offsets || !out->dst_row ||
         !out->src_index || !out->send_buf)
         return MOE_ERR_INVALID_ARG;
-    if (!logits || !x) return MOE_ERR_INVALID_ARG;
+    if (!x || (!logits && ctx->cfg.score_func != MOE_ROUTE_DENSE_TP)) return MOE_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(out->send_buf) || !aligned16(logits)) return MOE_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const Derived &d = ctx->d;

@@ -248,13 +248,40 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
         if (e < E && s_nlive[e] > 0) avail_mask |= 1u << q;
     }
 
+    // Dense-FFN mode (score_func 2): the "experts" are the k = TP shards of E/k replicated
+    // FFN groups; a group is healthy only if every shard is live.  List the healthy groups.
+    const bool dense = p.score_func == 2;
+    if (dense) {
+        if (tid == 0) {
+            int n = 0;
+            for (int g = 0; g < E / k; ++g) {
+                bool healthy = true;
+                for (int sh = 0; sh < k; ++sh) healthy = healthy && (s_nlive[g * k + sh] > 0);
+                if (healthy) s_lrank[n++] = g;             // s_lrank is free until the histogram step
+            }
+            s_warp_sums[0] = n;
+        }
+        __syncthreads();
+    }
+    const int n_healthy = dense ? s_warp_sums[0] : 0;
+
     // ---- a1..a6 per token -------------------------------------------------
     for (int lt0 = warp * kTokPerWarp; lt0 < tb; lt0 += kRouteWarps * kTokPerWarp) {
         const int lt = lt0 + sub;
         const int t = t0 + lt;
         int id = 0, slot = -1; float w = 0.0f;
         if (t0 + lt0 < p.T) {                            // warp-uniform: some token of the warp exists
-            route_tokens<EPL, LPT>(p, t0 + lt0, avail_mask, s_nlive, s_live, fallback_expert, id, w, slot);
+            if (dense) {
+                // tokens are dealt evenly over the healthy groups; each goes to all shards of its
+                // group with weight route_scale (the shards' partial results add up in combine)
+                if (sl < k && t < p.T) {
+                    id = s_lrank[t % n_healthy] * k + sl;
+                    w = p.route_scale;
+                    slot = s_live[id * p.max_rep + (t % s_nlive[id])];
+                }
+            } else {
+                route_tokens<EPL, LPT>(p, t0 + lt0, avail_mask, s_nlive, s_live, fallback_expert, id, w, slot);
+            }
             if (t >= p.T) slot = -1;
             if (sl < k && t < p.T) {
                 const size_t i = (size_t)t * k + sl;
