@@ -108,16 +108,18 @@ __device__ __forceinline__ float exp_spec(float z)
 
 __device__ __forceinline__ float sigmoid_spec(float x)
 {
-    return __fdiv_rn(1.0f, __fadd_rn(1.0f, exp_spec(-x)));
+    // 1 / d: the correctly rounded reciprocal is the correctly rounded quotient 1.0f / d
+    return __frcp_rn(__fadd_rn(1.0f, exp_spec(-x)));
 }
 
 // Order-preserving map from fp32 to uint32 (larger float <=> larger integer),
-// with -0 folded onto +0 so that equal floats get equal codes.  0 is below the
+// with -0 folded onto +0 (adding +0 in round-to-nearest turns -0 into +0 and
+// changes nothing else) so that equal floats get equal codes.  0 is below the
 // code of -inf and marks "already taken / not a candidate".
 __device__ __forceinline__ uint32_t key_code(float f)
 {
-    uint32_t u = (f == 0.0f) ? 0u : __float_as_uint(f);
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+    const uint32_t u = __float_as_uint(__fadd_rn(f, 0.0f));
+    return u ^ (static_cast<uint32_t>(static_cast<int32_t>(u) >> 31) | 0x80000000u);
 }
 constexpr uint32_t kCodeNegInf = 0x007FFFFFu;   // key_code(-inf)
 

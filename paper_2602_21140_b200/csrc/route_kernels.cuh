@@ -82,6 +82,7 @@ __device__ __forceinline__ void route_tokens(const RouteParams &p, int t_first, 
     const float *row = p.logits + (size_t)t * E;
     const float neg_inf = __int_as_float(0xff800000);
     const bool sigmoid = p.score_func != 0;
+    const bool grouped = p.n_group > 1;
 
     // a1 gate scores, a2 availability mask, and the two best keys of this lane (for a3)
     uint32_t code[EPL];
@@ -106,8 +107,10 @@ __device__ __forceinline__ void route_tokens(const RouteParams &p, int t_first, 
                     kf = __fadd_rn(sigmoid_spec(lg[u]), (e0 + q < E) ? __ldg(p.bias + e0 + q) : 0.0f);
                 const bool ok = ((avail_mask >> q) & 1u) && (lg[u] != neg_inf);
                 kf = ok ? kf : neg_inf;
-                if (kf > h1) { h2 = h1; h1 = kf; }
-                else if (kf > h2) { h2 = kf; }
+                if (grouped) {                            // running two best keys of the lane
+                    h2 = fmaxf(h2, fminf(h1, kf));
+                    h1 = fmaxf(h1, kf);
+                }
                 code[q] = key_code(kf);
             }
         }
@@ -151,13 +154,15 @@ __device__ __forceinline__ void route_tokens(const RouteParams &p, int t_first, 
         const int sel_e = __shfl_sync(full, e0 + lq, src, LPT);
         const bool bad = m <= kCodeNegInf;               // nothing selectable is left
         if (sl == j) { my_id = bad ? fallback_expert : sel_e; my_bad = bad; }
-        if (sl == src && !bad) {
-#pragma unroll
-            for (int q = 0; q < EPL; ++q) if (q == lq) code[q] = 0;
+        if (sl == src && !bad) {                         // drop the pick, find the lane's next best
+            const int taken = lq;
             lbest = 0; lq = 0;
 #pragma unroll
-            for (int q = 0; q < EPL; ++q)
-                if (code[q] > lbest) { lbest = code[q]; lq = q; }
+            for (int q = 0; q < EPL; ++q) {
+                const uint32_t c = (q == taken) ? 0u : code[q];
+                code[q] = c;
+                if (c > lbest) { lbest = c; lq = q; }
+            }
         }
     }
 
