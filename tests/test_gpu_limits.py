@@ -1,0 +1,87 @@
+"""GPU parity at the edges of the supported shapes: most experts, largest k,
+most replicas per expert, many slots, large routing tiles, tokens far below
+max_tokens."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2602_21140_b200 import binding as B
+from paper_2602_21140_b200 import workloads as W
+from gpu_util import assert_y_close, bf16_bits, check_dispatch, run_and_check, to_dev
+from util import oracle_cfg
+
+pytestmark = pytest.mark.gpu
+
+
+def _replicated_layout(E, R, S, copies):
+    """Copy c of expert e lives on rank (e + c * R / copies) mod R: `copies` distinct ranks each."""
+    assert E * copies == R * S and R % copies == 0
+    s2e = np.full(R * S, -1, np.int32)
+    used = [0] * R
+    for e in range(E):
+        for c in range(copies):
+            r = (e + c * (R // copies)) % R
+            s2e[r * S + used[r]] = e
+            used[r] += 1
+    return s2e
+
+
+@pytest.mark.parametrize("score", [W.SOFTMAX, W.SIGMOID])
+def test_most_experts_largest_k(score):
+    wl = W.Workload("wide", T=300, H=64, E=512, k=16, R=64, S=8, score_func=score, seed=41, max_replicas=1)
+    run_and_check(wl, W.make_inputs(wl), (3, 17))
+
+
+def test_grouped_at_512_experts():
+    wl = W.Workload("wide-grouped", T=200, H=64, E=512, k=8, R=64, S=8, score_func=W.SIGMOID,
+                    n_group=8, topk_group=4, seed=42, max_replicas=1)
+    run_and_check(wl, W.make_inputs(wl), (0, 63))
+
+
+def test_eight_replicas_per_expert_and_many_failures():
+    E, R, S = 32, 32, 8
+    wl = W.Workload("replicated", T=500, H=64, E=E, k=4, R=R, S=S, seed=43, max_replicas=8)
+    inp = W.make_inputs(dataclasses.replace(wl, max_replicas=1, R=4, S=8))     # logits / x / bias only
+    inp["slot_to_expert"] = _replicated_layout(E, R, S, 8)
+    inp["slot_scale"] = np.random.default_rng(2).uniform(0.5, 1.5, R * S).astype(np.float32)
+    for failed in [(), (1,), tuple(range(0, 32, 2)), tuple(range(1, 29))]:
+        if not oracle.failure_set_ok(oracle_cfg(wl), inp["slot_to_expert"], failed):
+            continue
+        out, _, ref = run_and_check(wl, inp, failed)
+        assert len(np.unique(ref["topk_slot"])) > wl.k       # replicas are actually spread over
+
+
+def test_many_slots():
+    wl = W.Workload("slots", T=400, H=64, E=256, k=8, R=128, S=8, seed=44, max_replicas=1)   # 1024 slots
+    inp = W.make_inputs(dataclasses.replace(wl, R=32, S=8))
+    s2e = np.full(wl.P, -1, np.int32)
+    s2e[::4] = np.arange(256)                                  # experts on every fourth slot
+    inp["slot_to_expert"] = s2e
+    inp["slot_scale"] = np.random.default_rng(3).uniform(0.5, 1.5, wl.P).astype(np.float32)
+    run_and_check(wl, inp, (5, 77))
+
+
+@pytest.mark.parametrize("max_tokens", [5000, 40000, 131072])
+def test_large_routing_tiles_and_partial_batches(max_tokens):
+    # the routing tile grows with max_tokens (64 ... 1024 tokens); batches far below it still work
+    wl = W.WORKLOADS["dsv3"]
+    for T in (1, 777, 4500):
+        inp = W.make_inputs(wl, T=T, H=64)
+        cfg = B.config_for_workload(wl, max_tokens=max_tokens, hidden=64)
+        router = B.MoeRouter(cfg, inp["slot_to_expert"], inp["bias"], inp["slot_scale"])
+        router.set_failed_ranks((7, 20))
+        run_and_check(wl, inp, (7, 20), router=router)
+        router.close()
+
+
+def test_config_limits_are_enforced():
+    wl = W.WORKLOADS["dsv3"]
+    for field, value in (("max_tokens", 262145), ("num_experts", 513), ("top_k", 17), ("max_replicas", 9)):
+        cfg = B.config_for_workload(wl)
+        setattr(cfg, field, value)
+        assert B.moe_workspace_bytes(cfg) == 0, field
+    cfg = B.config_for_workload(wl, max_tokens=262144)
+    assert B.moe_workspace_bytes(cfg) > 0
