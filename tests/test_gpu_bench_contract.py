@@ -1,0 +1,32 @@
+"""The benchmark's one-line JSON contract, checked on the tiny workload."""
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.mark.gpu
+def test_bench_prints_one_json_line_with_every_key():
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--workload", "tiny", "--steps", "20",
+                          "--warmup", "3"], capture_output=True, text=True, timeout=900, cwd=ROOT)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.strip()]
+    assert len(lines) == 1
+    r = json.loads(lines[0])
+    for key in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better",
+                "scaling", "vs_baseline", "dtype", "data", "config", "clocks", "e2e", "gpu_launches",
+                "roofline", "cpu_baseline", "remap"):
+        assert key in r, key
+    assert r["value"] > 0 and r["steps"] == 20 and r["n_gpus"] == 1 and r["scaling"] == "weak"
+    assert r["vs_baseline"] is None and r["data"] == "synthetic" and "workload" in r["config"]
+    assert r["gpu_launches"] >= 3 * 20
+    rf = r["roofline"]
+    assert rf["bound"] == "hbm" and rf["unit"] == "GB/s" and abs(rf["frac"] - rf["achieved"] / rf["peak"]) < 1e-9
+    assert rf["traffic"] is None                       # ncu traffic figures belong to the DSv3 shape only
+    assert r["cpu_baseline"]["kind"] == "oracle" and r["cpu_baseline"]["cores"] == 1
+    assert r["e2e"]["h2d_bytes_per_step"] > 0 and r["e2e"]["d2h_bytes_per_step"] > 0
+    assert r["remap"]["first_step_matches_oracle"] is True and r["remap"]["graph_recaptured"] is False
