@@ -34,8 +34,9 @@ METRIC = "dispatch+combine tokens/s at DSv3 shape"
 UNIT = "tokens/s"
 
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from ncu captures of
-# the kernels as they stand; None when a kernel changed after its last capture.
-NCU_TRAFFIC_BYTES = {"k_scatter": 998_323_200, "k_combine": 1_050_063_616}   # profiles/k_*_dsv3.md
+# the kernels as they stand at the DSv3 shape (summaries under profiles/); None when a kernel
+# changed after its last capture.
+NCU_TRAFFIC_BYTES = {"k_scatter": 998_323_200, "k_combine": 1_050_063_616}
 
 
 def env_rank():
@@ -53,7 +54,9 @@ def measured_peaks():
 
 
 def algorithmic_bytes(wl, T):
-    """Bytes the method must move per launch, by kernel."""
+    """Bytes the method must move per launch, by kernel: routing reads the logits and writes
+    four index/weight words per assignment; scatter reads each row once and writes it k times;
+    combine reads k rows and writes one (plus the small index traffic of each)."""
     row = 2 * wl.H
     route = T * (4 * wl.E + 16 * wl.k)                 # logits in; ids, weights, slots, ranks out
     scatter = T * ((1 + wl.k) * row + 20 * wl.k)       # x once, k copies out; slot/rank/offset in, rows out
