@@ -161,6 +161,7 @@ __global__ void __launch_bounds__(kCombineBulkMaxWarps * 32) k_combine_bulk(Comb
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncwarp();
+    pdl_enter();                                           // the ring is set up; now wait for the inputs
 
     const int chunks = (p.hv + kChunkV - 1) / kChunkV;
     const long long items = (long long)p.T * chunks;

@@ -23,6 +23,15 @@ struct Control {
     int pad;
 };
 
+// Programmatic dependent launch: let the next kernel of the stream be scheduled while this
+// one is still running, and hold this kernel until the previous one has completed and its
+// memory is visible.  Both are no-ops for a kernel launched without the attribute.
+__device__ __forceinline__ void pdl_enter()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 __device__ __forceinline__ unsigned lane_id() { return threadIdx.x & 31u; }
 
 __device__ __forceinline__ unsigned lanemask_lt()

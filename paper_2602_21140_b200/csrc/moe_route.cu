@@ -249,6 +249,23 @@ size_t device_bytes_for(const Derived &d, int max_tokens)
     return b;
 }
 
+// Launch with the programmatic-dependent-launch attribute (when `pdl`), so that the kernel's
+// blocks can be scheduled while the previous kernel of the stream drains.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                          bool pdl, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
+bool g_pdl = true;      // set once per context from MOE_PDL
+
 template <int EPL, int LPT>
 cudaError_t launch_route_t(const RouteParams &p, int tiles, size_t smem, cudaStream_t st)
 {
@@ -257,8 +274,7 @@ cudaError_t launch_route_t(const RouteParams &p, int tiles, size_t smem, cudaStr
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
-    k_route<EPL, LPT><<<tiles, kRouteThreads, smem, st>>>(p);
-    return cudaGetLastError();
+    return launch_kernel(k_route<EPL, LPT>, dim3(tiles), dim3(kRouteThreads), smem, st, g_pdl, p);
 }
 
 template <int LPT>
@@ -453,6 +469,7 @@ moe_status moe_route_init(const moe_config *cfg, const int32_t *slot_to_expert, 
     }
     if (ok) {
         ctx->route_smem = route_smem_bytes(d.E, d.max_rep, d.tokens_per_block, d.k, d.P);
+        g_pdl = env_int("MOE_PDL", 1) != 0;
         ctx->scatter_impl = env_int("MOE_SCATTER_IMPL", 0);
         ctx->bulk_stages = std::min(8, std::max(1, env_int("MOE_BULK_STAGES", 4)));
         const size_t stage_bytes = ((size_t)d.H * 2 + 127) & ~(size_t)127;
@@ -676,11 +693,11 @@ moe_status moe_dispatch(moe_ctx *ctx, const float *logits, const void *x, int32_
         const long long want = (items + kScatterThreads / 32 - 1) / (kScatterThreads / 32);
         const int grid = (int)std::min<long long>(want, (long long)ctx->sm_count * ctx->scatter_blocks_per_sm);
         switch (un) {
-            case 8: k_scatter_vec<8><<<grid, kScatterThreads, 0, st>>>(sp); break;
-            case 16: k_scatter_vec<16><<<grid, kScatterThreads, 0, st>>>(sp); break;
-            case 28: k_scatter_vec<28><<<grid, kScatterThreads, 0, st>>>(sp); break;
-            case 32: k_scatter_vec<32><<<grid, kScatterThreads, 0, st>>>(sp); break;
-            default: k_scatter_vec<4><<<grid, kScatterThreads, 0, st>>>(sp); break;
+            case 8: launch_kernel(k_scatter_vec<8>, dim3(grid), dim3(kScatterThreads), 0, st, g_pdl, sp); break;
+            case 16: launch_kernel(k_scatter_vec<16>, dim3(grid), dim3(kScatterThreads), 0, st, g_pdl, sp); break;
+            case 28: launch_kernel(k_scatter_vec<28>, dim3(grid), dim3(kScatterThreads), 0, st, g_pdl, sp); break;
+            case 32: launch_kernel(k_scatter_vec<32>, dim3(grid), dim3(kScatterThreads), 0, st, g_pdl, sp); break;
+            default: launch_kernel(k_scatter_vec<4>, dim3(grid), dim3(kScatterThreads), 0, st, g_pdl, sp); break;
         }
     }
     if (cudaGetLastError() != cudaSuccess) return MOE_ERR_CUDA;
@@ -707,11 +724,11 @@ moe_status moe_combine(moe_ctx *ctx, const void *expert_buf, int32_t T, void *y,
         const long long want = (items + nw - 1) / nw;
         const int grid = (int)std::min<long long>(want, (long long)ctx->sm_count * ctx->combine_ctas_per_sm);
         if (ctx->combine_u == 1)
-            k_combine_bulk<1><<<grid, nw * 32, ctx->combine_smem, st>>>(cp, ctx->combine_stages, ctx->d_ctl);
+            launch_kernel(k_combine_bulk<1>, dim3(grid), dim3(nw * 32), ctx->combine_smem, st, g_pdl, cp, ctx->combine_stages, ctx->d_ctl);
         else if (ctx->combine_u == 2)
-            k_combine_bulk<2><<<grid, nw * 32, ctx->combine_smem, st>>>(cp, ctx->combine_stages, ctx->d_ctl);
+            launch_kernel(k_combine_bulk<2>, dim3(grid), dim3(nw * 32), ctx->combine_smem, st, g_pdl, cp, ctx->combine_stages, ctx->d_ctl);
         else
-            k_combine_bulk<4><<<grid, nw * 32, ctx->combine_smem, st>>>(cp, ctx->combine_stages, ctx->d_ctl);
+            launch_kernel(k_combine_bulk<4>, dim3(grid), dim3(nw * 32), ctx->combine_smem, st, g_pdl, cp, ctx->combine_stages, ctx->d_ctl);
         return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
     }
     const int chunks = (cp.hv + kCombineChunk - 1) / kCombineChunk;

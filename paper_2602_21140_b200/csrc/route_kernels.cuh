@@ -213,6 +213,7 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned full = 0xffffffffu;
 
+    pdl_enter();
     if (tid == 0) {
         s_epoch = ld_relaxed_u32(&p.ctl->epoch);
         s_ticket = atomicAdd(&p.ctl->ticket, 1u);

@@ -51,6 +51,7 @@ __global__ void __launch_bounds__(kScatterThreads) k_scatter_vec(ScatterParams p
 {
     constexpr int kChunk = 32 * UNROLL;
     const unsigned full = 0xffffffffu;
+    pdl_enter();
     const int lane = lane_id();
     const int chunks = (p.hv + kChunk - 1) / kChunk;
     const long long items = (long long)p.T * chunks;
