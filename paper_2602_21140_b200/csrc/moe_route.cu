@@ -220,6 +220,7 @@ struct moe_ctx {
     bool stage_used[kStagingSlots];
     unsigned stage_next;
     // launch choices
+    bool pdl;              // launch with the programmatic-dependent-launch attribute
     int scatter_impl;      // 0 = vector, 1 = bulk copies
     int bulk_stages, bulk_ctas_per_sm;
     int scatter_blocks_per_sm, combine_blocks_per_sm, scatter_unroll;
@@ -264,44 +265,43 @@ cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_
     return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
-bool g_pdl = true;      // set once per context from MOE_PDL
-
 template <int EPL, int LPT>
-cudaError_t launch_route_t(const RouteParams &p, int tiles, size_t smem, cudaStream_t st)
+cudaError_t launch_route_t(const RouteParams &p, int tiles, size_t smem, cudaStream_t st, bool pdl)
 {
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(k_route<EPL, LPT>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
-    return launch_kernel(k_route<EPL, LPT>, dim3(tiles), dim3(kRouteThreads), smem, st, g_pdl, p);
+    return launch_kernel(k_route<EPL, LPT>, dim3(tiles), dim3(kRouteThreads), smem, st, pdl, p);
 }
 
 template <int LPT>
-cudaError_t launch_route_lpt(int epl, const RouteParams &p, int tiles, size_t smem, cudaStream_t st)
+cudaError_t launch_route_lpt(int epl, const RouteParams &p, int tiles, size_t smem, cudaStream_t st, bool pdl)
 {
     switch (epl) {
-        case 1: return launch_route_t<1, LPT>(p, tiles, smem, st);
-        case 2: return launch_route_t<2, LPT>(p, tiles, smem, st);
-        case 3: return launch_route_t<3, LPT>(p, tiles, smem, st);
-        case 4: return launch_route_t<4, LPT>(p, tiles, smem, st);
-        case 5: return launch_route_t<5, LPT>(p, tiles, smem, st);
-        case 6: return launch_route_t<6, LPT>(p, tiles, smem, st);
-        case 8: return launch_route_t<8, LPT>(p, tiles, smem, st);
-        case 10: return launch_route_t<10, LPT>(p, tiles, smem, st);
-        case 12: return launch_route_t<12, LPT>(p, tiles, smem, st);
-        case 16: return launch_route_t<16, LPT>(p, tiles, smem, st);
-        case 20: return launch_route_t<20, LPT>(p, tiles, smem, st);
-        case 24: return launch_route_t<24, LPT>(p, tiles, smem, st);
-        case 32: return launch_route_t<32, LPT>(p, tiles, smem, st);
+        case 1: return launch_route_t<1, LPT>(p, tiles, smem, st, pdl);
+        case 2: return launch_route_t<2, LPT>(p, tiles, smem, st, pdl);
+        case 3: return launch_route_t<3, LPT>(p, tiles, smem, st, pdl);
+        case 4: return launch_route_t<4, LPT>(p, tiles, smem, st, pdl);
+        case 5: return launch_route_t<5, LPT>(p, tiles, smem, st, pdl);
+        case 6: return launch_route_t<6, LPT>(p, tiles, smem, st, pdl);
+        case 8: return launch_route_t<8, LPT>(p, tiles, smem, st, pdl);
+        case 10: return launch_route_t<10, LPT>(p, tiles, smem, st, pdl);
+        case 12: return launch_route_t<12, LPT>(p, tiles, smem, st, pdl);
+        case 16: return launch_route_t<16, LPT>(p, tiles, smem, st, pdl);
+        case 20: return launch_route_t<20, LPT>(p, tiles, smem, st, pdl);
+        case 24: return launch_route_t<24, LPT>(p, tiles, smem, st, pdl);
+        case 32: return launch_route_t<32, LPT>(p, tiles, smem, st, pdl);
     }
     return cudaErrorInvalidValue;
 }
 
-cudaError_t launch_route(int epl, int lpt, const RouteParams &p, int tiles, size_t smem, cudaStream_t st)
+cudaError_t launch_route(int epl, int lpt, const RouteParams &p, int tiles, size_t smem, cudaStream_t st,
+                         bool pdl)
 {
-    if (lpt == 8) return launch_route_lpt<8>(epl, p, tiles, smem, st);
-    if (lpt == 16) return launch_route_lpt<16>(epl, p, tiles, smem, st);
+    if (lpt == 8) return launch_route_lpt<8>(epl, p, tiles, smem, st, pdl);
+    if (lpt == 16) return launch_route_lpt<16>(epl, p, tiles, smem, st, pdl);
     return cudaErrorInvalidValue;
 }
 
@@ -469,7 +469,7 @@ moe_status moe_route_init(const moe_config *cfg, const int32_t *slot_to_expert, 
     }
     if (ok) {
         ctx->route_smem = route_smem_bytes(d.E, d.max_rep, d.tokens_per_block, d.k, d.P);
-        g_pdl = env_int("MOE_PDL", 1) != 0;
+        ctx->pdl = env_int("MOE_PDL", 1) != 0;
         ctx->scatter_impl = env_int("MOE_SCATTER_IMPL", 0);
         ctx->bulk_stages = std::min(8, std::max(1, env_int("MOE_BULK_STAGES", 4)));
         const size_t stage_bytes = ((size_t)d.H * 2 + 127) & ~(size_t)127;
@@ -673,7 +673,7 @@ moe_status moe_dispatch(moe_ctx *ctx, const float *logits, const void *x, int32_
     rp.rank_counts = out->rank_counts; rp.rank_offsets = out->rank_offsets;
     rp.desc = ctx->d_desc; rp.ctl = ctx->d_ctl;
     const int tiles = (T + d.tokens_per_block - 1) / d.tokens_per_block;
-    if (launch_route(d.epl, d.lpt, rp, tiles, ctx->route_smem, st) != cudaSuccess) return MOE_ERR_CUDA;
+    if (launch_route(d.epl, d.lpt, rp, tiles, ctx->route_smem, st, ctx->pdl) != cudaSuccess) return MOE_ERR_CUDA;
     if (ctx->timing_event && cudaEventRecord(ctx->timing_event, st) != cudaSuccess) return MOE_ERR_CUDA;
 
     ScatterParams sp;
@@ -693,11 +693,11 @@ moe_status moe_dispatch(moe_ctx *ctx, const float *logits, const void *x, int32_
         const long long want = (items + kScatterThreads / 32 - 1) / (kScatterThreads / 32);
         const int grid = (int)std::min<long long>(want, (long long)ctx->sm_count * ctx->scatter_blocks_per_sm);
         switch (un) {
-            case 8: launch_kernel(k_scatter_vec<8>, dim3(grid), dim3(kScatterThreads), 0, st, g_pdl, sp); break;
-            case 16: launch_kernel(k_scatter_vec<16>, dim3(grid), dim3(kScatterThreads), 0, st, g_pdl, sp); break;
-            case 28: launch_kernel(k_scatter_vec<28>, dim3(grid), dim3(kScatterThreads), 0, st, g_pdl, sp); break;
-            case 32: launch_kernel(k_scatter_vec<32>, dim3(grid), dim3(kScatterThreads), 0, st, g_pdl, sp); break;
-            default: launch_kernel(k_scatter_vec<4>, dim3(grid), dim3(kScatterThreads), 0, st, g_pdl, sp); break;
+            case 8: launch_kernel(k_scatter_vec<8>, dim3(grid), dim3(kScatterThreads), 0, st, ctx->pdl, sp); break;
+            case 16: launch_kernel(k_scatter_vec<16>, dim3(grid), dim3(kScatterThreads), 0, st, ctx->pdl, sp); break;
+            case 28: launch_kernel(k_scatter_vec<28>, dim3(grid), dim3(kScatterThreads), 0, st, ctx->pdl, sp); break;
+            case 32: launch_kernel(k_scatter_vec<32>, dim3(grid), dim3(kScatterThreads), 0, st, ctx->pdl, sp); break;
+            default: launch_kernel(k_scatter_vec<4>, dim3(grid), dim3(kScatterThreads), 0, st, ctx->pdl, sp); break;
         }
     }
     if (cudaGetLastError() != cudaSuccess) return MOE_ERR_CUDA;
@@ -724,11 +724,11 @@ moe_status moe_combine(moe_ctx *ctx, const void *expert_buf, int32_t T, void *y,
         const long long want = (items + nw - 1) / nw;
         const int grid = (int)std::min<long long>(want, (long long)ctx->sm_count * ctx->combine_ctas_per_sm);
         if (ctx->combine_u == 1)
-            launch_kernel(k_combine_bulk<1>, dim3(grid), dim3(nw * 32), ctx->combine_smem, st, g_pdl, cp, ctx->combine_stages, ctx->d_ctl);
+            launch_kernel(k_combine_bulk<1>, dim3(grid), dim3(nw * 32), ctx->combine_smem, st, ctx->pdl, cp, ctx->combine_stages, ctx->d_ctl);
         else if (ctx->combine_u == 2)
-            launch_kernel(k_combine_bulk<2>, dim3(grid), dim3(nw * 32), ctx->combine_smem, st, g_pdl, cp, ctx->combine_stages, ctx->d_ctl);
+            launch_kernel(k_combine_bulk<2>, dim3(grid), dim3(nw * 32), ctx->combine_smem, st, ctx->pdl, cp, ctx->combine_stages, ctx->d_ctl);
         else
-            launch_kernel(k_combine_bulk<4>, dim3(grid), dim3(nw * 32), ctx->combine_smem, st, g_pdl, cp, ctx->combine_stages, ctx->d_ctl);
+            launch_kernel(k_combine_bulk<4>, dim3(grid), dim3(nw * 32), ctx->combine_smem, st, ctx->pdl, cp, ctx->combine_stages, ctx->d_ctl);
         return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
     }
     const int chunks = (cp.hv + kCombineChunk - 1) / kCombineChunk;
