@@ -57,9 +57,14 @@ typedef enum {
 enum { MOE_SCORE_SOFTMAX = 0, MOE_SCORE_SIGMOID = 1, MOE_ROUTE_DENSE_TP = 2 };
 
 /* Limits of this build: num_experts <= 512, top_k <= 16, max_replicas <= 8,
- * num_ranks*slots_per_rank <= 4096, hidden % 8 == 0.  With n_group > 1:
- * num_experts % n_group == 0, top_k % topk_group == 0 and top_k/topk_group
- * in {1, 2}. */
+ * num_ranks*slots_per_rank <= 4096 (and small enough for the routing kernel's
+ * shared-memory tables, about 2000 slots at 512 experts), max_tokens <= 262144,
+ * max_tokens*top_k < 2^30, hidden % 8 == 0.  With n_group > 1:
+ * num_experts % n_group == 0, top_k % topk_group == 0, top_k/topk_group in
+ * {1, 2}, and the experts of a group must map onto a power-of-two run of lanes
+ * (any group size that is a power of two, or a multiple of one of
+ * 1,2,3,4,5,6,8,10,12,16,20,24,32 by a power of two, qualifies).  A shape outside
+ * these limits makes moe_route_init return MOE_ERR_INVALID_ARG. */
 typedef struct {
     int32_t num_experts;    /* E: logical experts                                            */
     int32_t top_k;          /* k: experts per token                                          */
@@ -268,7 +273,8 @@ moe_status moe_plan_routing_state(const moe_config *cfg, const int32_t *slot_to_
  *   slot_counts  device [P]   i32 out   slot_offsets device [P+1] i32 out
  *   rank_counts  device [R]   i32 out   rank_offsets device [R+1] i32 out
  *   dst_row      device [n_assign] i32 out   src_index device [n_assign] i32 out
- * with P = num_ranks * slots_per_rank; meanings as in moe_dispatch_out.
+ * with P = num_ranks * slots_per_rank; meanings as in moe_dispatch_out, ranks in their
+ * physical numbering (this entry point knows no rank order).
  *
  * Limits: P <= 512 and n_assign <= 262144; anything larger returns
  * MOE_ERR_CAPACITY and launches nothing.  n_assign = 0 writes zero counts.
