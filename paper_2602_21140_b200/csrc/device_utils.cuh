@@ -100,7 +100,11 @@ __device__ __forceinline__ void st_stream_v4(uint4 *p, const uint4 &v)
 __device__ __forceinline__ float exp_spec(float z)
 {
     z = fminf(fmaxf(z, -87.0f), 88.0f);
-    const float n = rintf(__fmul_rn(z, 0x1.715476p+0f));
+    // rint by adding and removing 1.5 * 2^23: at that magnitude one ulp is 1, so the add rounds
+    // z*log2e (|.| < 128) to the nearest integer, ties to even, and the subtraction is exact.
+    // The integer itself sits in the low mantissa bits of the biased sum.
+    const float biased = __fadd_rn(__fmul_rn(z, 0x1.715476p+0f), 12582912.0f);
+    const float n = __fsub_rn(biased, 12582912.0f);
     float r = __fmaf_rn(-n, 0x1.62e430p-1f, z);
     r = __fmaf_rn(-n, -0x1.05c610p-29f, r);
     float p = 0x1.a01a02p-13f;
@@ -111,7 +115,7 @@ __device__ __forceinline__ float exp_spec(float z)
     p = __fmaf_rn(p, r, 0.5f);
     p = __fmaf_rn(p, r, 1.0f);
     p = __fmaf_rn(p, r, 1.0f);
-    const float two_n = __int_as_float((static_cast<int>(n) + 127) << 23);
+    const float two_n = __int_as_float((__float_as_int(biased) << 23) + 0x3f800000);   // (n + 127) << 23
     return __fmul_rn(p, two_n);
 }
 

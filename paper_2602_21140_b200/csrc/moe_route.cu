@@ -496,7 +496,11 @@ moe_status moe_route_init(const moe_config *cfg, const int32_t *slot_to_expert, 
         }
         ctx->combine_blocks_per_sm = std::max(1, env_int("MOE_COMBINE_BLOCKS_PER_SM", 8));
         ctx->combine_impl = env_int("MOE_COMBINE_IMPL", 1);
-        ctx->combine_u = env_int("MOE_COMBINE_U", 1);
+        // a ring stage holds one column chunk of all k rows: widen the chunk for small k so that a
+        // stage stays near 4 KB and the ring keeps as many bytes in flight as with k = 8
+        int u_auto = d.k <= 2 ? 4 : (d.k <= 4 ? 2 : 1);
+        while (u_auto > 1 && 32 * u_auto > d.H / 8) u_auto /= 2;        // never wider than a row
+        ctx->combine_u = env_int("MOE_COMBINE_U", u_auto);
         if (ctx->combine_u != 1 && ctx->combine_u != 2 && ctx->combine_u != 4) ctx->combine_u = 2;
         ctx->combine_warps = std::min(kCombineBulkMaxWarps, std::max(1, env_int("MOE_COMBINE_WARPS", 8)));
         ctx->combine_stages = std::min(8, std::max(2, env_int("MOE_COMBINE_STAGES", 3)));

@@ -64,6 +64,27 @@ __host__ __device__ inline size_t route_smem_bytes(int E, int max_rep, int token
     return words * sizeof(int32_t) + (size_t)kRouteWarps * P * sizeof(uint16_t);
 }
 
+// Block B (experts 4B..4B+3 of a lane) lost element `taken`: blank it and find the block's
+// next best code, lowest index first among equals.
+template <int B, int EPL>
+__device__ __forceinline__ void rescan_block(uint32_t (&code)[EPL], uint32_t (&bm)[(EPL + 3) / 4],
+                                             int (&bq)[(EPL + 3) / 4], int taken)
+{
+    if constexpr (4 * B < EPL) {
+        uint32_t best = 0; int at = 4 * B;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            constexpr int q0 = 4 * B;
+            if (q0 + u < EPL) {
+                const uint32_t c = (q0 + u == taken) ? 0u : code[q0 + u];
+                code[q0 + u] = c;
+                if (c > best) { best = c; at = q0 + u; }
+            }
+        }
+        bm[B] = best; bq[B] = at;
+    }
+}
+
 // Route 32/LPT tokens with one warp.  Lanes [sub*LPT, (sub+1)*LPT) own token
 // t_first + sub.  On return, sub-lane j < k of a token holds its j-th chosen
 // expert, the weight and the physical slot.
@@ -136,33 +157,49 @@ __device__ __forceinline__ void route_tokens(const RouteParams &p, int t_first, 
         active = (g < p.n_group) && (rank < p.topk_group);
     }
 
-    // a4 top-k: k rounds of arg-max over order-preserving integer codes
-    uint32_t lbest = 0; int lq = 0;
-    if (active) {
+    // a4 top-k: k rounds of arg-max over order-preserving integer codes.  A lane keeps the best
+    // code of each block of four of its experts, so that after a pick only the block that lost
+    // an element is scanned again (the rounds are bound by instruction issue).
+    constexpr int kBlocks = (EPL + 3) / 4;
+    uint32_t bm[kBlocks]; int bq[kBlocks];
 #pragma unroll
-        for (int q = 0; q < EPL; ++q)
-            if (code[q] > lbest) { lbest = code[q]; lq = q; }
+    for (int b = 0; b < kBlocks; ++b) {
+        bm[b] = 0; bq[b] = 4 * b;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int q = 4 * b + u;
+            if (q < EPL && active && code[q] > bm[b]) { bm[b] = code[q]; bq[b] = q; }
+        }
     }
+    uint32_t lbest = 0; int lq = 0;
+#pragma unroll
+    for (int b = 0; b < kBlocks; ++b)
+        if (bm[b] > lbest) { lbest = bm[b]; lq = bq[b]; }
+    const unsigned seg_mask = ((LPT == 32) ? 0xffffffffu : ((1u << LPT) - 1u)) << (sub * LPT);
     int my_id = fallback_expert; bool my_bad = false;
     for (int j = 0; j < p.k; ++j) {
-        uint32_t m = lbest;
-#pragma unroll
-        for (int off = LPT / 2; off > 0; off >>= 1) m = max(m, __shfl_xor_sync(full, m, off, LPT));
+        const uint32_t m = __reduce_max_sync(seg_mask, lbest);
         const unsigned ball = __ballot_sync(full, lbest == m);
-        const unsigned seg = (ball >> (sub * LPT)) & ((LPT == 32) ? 0xffffffffu : ((1u << LPT) - 1u));
-        const int src = __ffs(seg) - 1;                  // lowest lane = lowest expert id
+        const int src = __ffs(ball & seg_mask) - 1 - sub * LPT;   // lowest lane = lowest expert id
         const int sel_e = __shfl_sync(full, e0 + lq, src, LPT);
         const bool bad = m <= kCodeNegInf;               // nothing selectable is left
         if (sl == j) { my_id = bad ? fallback_expert : sel_e; my_bad = bad; }
         if (sl == src && !bad) {                         // drop the pick, find the lane's next best
             const int taken = lq;
+            switch (taken >> 2) {
+                case 0: rescan_block<0, EPL>(code, bm, bq, taken); break;
+                case 1: rescan_block<1, EPL>(code, bm, bq, taken); break;
+                case 2: rescan_block<2, EPL>(code, bm, bq, taken); break;
+                case 3: rescan_block<3, EPL>(code, bm, bq, taken); break;
+                case 4: rescan_block<4, EPL>(code, bm, bq, taken); break;
+                case 5: rescan_block<5, EPL>(code, bm, bq, taken); break;
+                case 6: rescan_block<6, EPL>(code, bm, bq, taken); break;
+                default: rescan_block<7, EPL>(code, bm, bq, taken); break;
+            }
             lbest = 0; lq = 0;
 #pragma unroll
-            for (int q = 0; q < EPL; ++q) {
-                const uint32_t c = (q == taken) ? 0u : code[q];
-                code[q] = c;
-                if (c > lbest) { lbest = c; lq = q; }
-            }
+            for (int b = 0; b < kBlocks; ++b)
+                if (bm[b] > lbest) { lbest = bm[b]; lq = bq[b]; }
         }
     }
 
