@@ -210,6 +210,91 @@ moe_status moe_dispatch(moe_ctx *ctx, const float *logits, const void *x, int32_
 moe_status moe_combine(moe_ctx *ctx, const void *expert_buf, int32_t T, void *y, void *cuda_stream);
 
 /*
+ * ---- Expert parallelism over several GPUs -----------------------------------
+ * Sec. 2.3: "dispatch" routes tokens to their experts and "combine" brings the expert
+ * outputs back; between real devices both are all-to-all exchanges (attention2expert /
+ * expert2attention).  Here the exchange is part of the kernels: the scatter stores each
+ * row straight into the receive buffer of the GPU that hosts the chosen slot, and the
+ * combine reads its k rows from those buffers, through pointers that are valid on the
+ * calling GPU (peer mappings).  No send buffer and no separate all-to-all exist.
+ *
+ * Group of `world` GPUs, one context per GPU, all built from the same moe_config,
+ * placement and failure state.  GPU d hosts the simulated ranks
+ * [d*R/world, (d+1)*R/world), i.e. the slots [d*spg, (d+1)*spg) with spg = P/world
+ * (num_ranks % world == 0).  Receive buffer of GPU d, bf16 [recv_rows, H]: the rows of
+ * its slots in ascending slot order; inside a slot the rows sent by GPU 0 first, then
+ * GPU 1, ..., each sender's rows in its own stable order (ascending i = t*k + j).
+ *
+ * One step on every GPU g, all on its stream:
+ *   moe_ep_route(logits_g)            -> out.topk_*, out.slot_counts = counts[g][:]
+ *   all-gather of slot_counts         -> counts_all device [world][P]   (caller: NCCL or any other way)
+ *   moe_ep_scatter(x_g, counts_all)   -> rows land in the owners' receive buffers; out.dst_row[i] =
+ *                                        row of assignment i in its owner's buffer;
+ *                                        recv_slot_offsets = layout of g's own receive buffer
+ *   (all GPUs' scatters must have completed before anyone reads a receive buffer: order the
+ *    streams with a collective or events; the experts then work on the receive buffers in place)
+ *   moe_ep_combine(y_g)               -> y[t,:] as in moe_combine, rows fetched from the owners
+ *   (all combines must have completed before the next step's scatter overwrites the buffers)
+ * The rank order must be the physical one (no moe_set_rank_order) in this mode.
+ */
+typedef struct {
+    int32_t world;            /* GPUs in the group                                              */
+    int32_t rank;             /* index of the calling GPU, 0 <= rank < world                    */
+    void *const *recv_bufs;   /* host [world]: device pointers, usable from the calling GPU, to
+                                 every GPU's receive buffer (own buffer at [rank]); 16-byte aligned */
+    int64_t recv_rows;        /* rows every receive buffer can hold (world*max_tokens*top_k always suffices) */
+} moe_ep_group;
+
+/*
+ * moe_ep_attach — bind a context to its group: copies the pointer table to the device and
+ * allocates the per-slot offset scratch (the only allocation of this mode; call it at
+ * set-up, not while capturing).  May be called again with other buffers.
+ * INVALID_ARG if num_ranks % world != 0, a pointer is NULL or misaligned, a rank order is
+ * set, or the shape leaves no room for the bulk-copy combine.
+ */
+moe_status moe_ep_attach(moe_ctx *ctx, const moe_ep_group *group, void *cuda_stream);
+
+/*
+ * moe_ep_route — the routing half of a dispatch (Sec. 2.1, Sec. 3.4 masking) for this GPU's
+ * T tokens: writes out->topk_ids / topk_weights / topk_slot and out->slot_counts (this
+ * GPU's assignments per physical slot, the row counts[rank][:] of the exchange).
+ * slot_offsets / rank_counts / rank_offsets describe this GPU's own assignments only;
+ * send_buf and src_index are not used and may be NULL.  T = 0 writes zero counts.
+ */
+moe_status moe_ep_route(moe_ctx *ctx, const float *logits, int32_t T, const moe_dispatch_out *out,
+                        void *cuda_stream);
+
+/*
+ * moe_ep_scatter — the dispatch exchange (Sec. 2.3, attention2expert).
+ *   x                 device [T,H] bf16, 16-byte aligned
+ *   counts_all        device [world][P] i32: slot_counts of every GPU after the all-gather
+ *   recv_slot_offsets device [P/world + 1] i32 out: first row of each of this GPU's slots in
+ *                     its own receive buffer, last entry = rows received
+ * Writes out->dst_row of the preceding moe_ep_route.  If the rows sent to a GPU exceed
+ * recv_rows the surplus rows are not written and that GPU's device status becomes
+ * MOE_ERR_CAPACITY (moe_get_device_status).  Allocates nothing, does not synchronise.
+ */
+moe_status moe_ep_scatter(moe_ctx *ctx, const void *x, int32_t T, const int32_t *counts_all,
+                          int32_t *recv_slot_offsets, void *cuda_stream);
+
+/*
+ * moe_ep_combine — the combine exchange (Sec. 2.3, expert2attention): as moe_combine, with
+ * row dst_row[t*k+j] read from the receive buffer of the GPU hosting topk_slot[t,j].
+ *   y device [T,H] bf16, 16-byte aligned
+ */
+moe_status moe_ep_combine(moe_ctx *ctx, int32_t T, void *y, void *cuda_stream);
+
+/*
+ * moe_ep_plan_host — the layout arithmetic of the exchange on the host, no CUDA call.
+ *   counts_all host [world][num_slots]
+ *   src_base   host [num_slots] out (or NULL): first row, in the owner's buffer, of `rank`'s rows for each slot
+ *   recv_slot_offsets host [num_slots/world + 1] out (or NULL): layout of `rank`'s own buffer
+ * CAPACITY if an offset exceeds 2^31 - 1.
+ */
+moe_status moe_ep_plan_host(const int32_t *counts_all, int32_t world, int32_t rank, int32_t num_slots,
+                            int32_t *src_base, int32_t *recv_slot_offsets);
+
+/*
  * moe_step_host — one dispatch + combine fed from HOST memory, for callers
  * that hold activations on the CPU: copies logits and x to the given device
  * staging buffers, runs moe_dispatch and moe_combine (expert_buf = the send

@@ -40,6 +40,7 @@ EXPORTED_SYMBOLS = (
     "moe_combine", "moe_step_host", "moe_set_timing_event", "moe_get_device_status", "moe_plan_routing_state",
     "moe_workspace_bytes", "moe_route_destroy", "moe_status_string", "moe_permute_static",
     "moe_set_failed_experts", "moe_compact_ranks", "moe_set_rank_order",
+    "moe_ep_attach", "moe_ep_route", "moe_ep_scatter", "moe_ep_combine", "moe_ep_plan_host",
 )
 
 
@@ -64,6 +65,11 @@ class moe_dispatch_out(ctypes.Structure):
                 ("slot_offsets", ctypes.c_void_p), ("rank_counts", ctypes.c_void_p),
                 ("rank_offsets", ctypes.c_void_p), ("dst_row", ctypes.c_void_p),
                 ("src_index", ctypes.c_void_p), ("send_buf", ctypes.c_void_p)]
+
+
+class moe_ep_group(ctypes.Structure):
+    _fields_ = [("world", ctypes.c_int32), ("rank", ctypes.c_int32),
+                ("recv_bufs", ctypes.POINTER(ctypes.c_void_p)), ("recv_rows", ctypes.c_int64)]
 
 
 def library_path() -> str:
@@ -110,6 +116,16 @@ def _lib():
         lib.moe_route_destroy.argtypes = [vp]
         lib.moe_permute_static.restype = ctypes.c_int
         lib.moe_permute_static.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+        lib.moe_ep_attach.restype = ctypes.c_int
+        lib.moe_ep_attach.argtypes = [vp, ctypes.POINTER(moe_ep_group), vp]
+        lib.moe_ep_route.restype = ctypes.c_int
+        lib.moe_ep_route.argtypes = [vp, vp, i32, ctypes.POINTER(moe_dispatch_out), vp]
+        lib.moe_ep_scatter.restype = ctypes.c_int
+        lib.moe_ep_scatter.argtypes = [vp, vp, i32, vp, vp, vp]
+        lib.moe_ep_combine.restype = ctypes.c_int
+        lib.moe_ep_combine.argtypes = [vp, i32, vp, vp]
+        lib.moe_ep_plan_host.restype = ctypes.c_int
+        lib.moe_ep_plan_host.argtypes = [vp, i32, i32, i32, vp, vp]
         lib.moe_status_string.restype = ctypes.c_char_p
         lib.moe_status_string.argtypes = [ctypes.c_int]
         _lib_handle = lib
@@ -245,6 +261,40 @@ def moe_permute_static(topk_slot_ptr: int, n_assign: int, num_ranks: int, slots_
                                      vp(cuda_stream))
 
 
+def moe_ep_attach(ctx, world: int, rank: int, recv_buf_ptrs, recv_rows: int, cuda_stream: int = 0) -> int:
+    """recv_buf_ptrs: `world` raw device addresses, usable from the calling GPU."""
+    ptrs = (ctypes.c_void_p * max(world, 1))(*[int(a) for a in recv_buf_ptrs])
+    group = moe_ep_group(world, rank, ctypes.cast(ptrs, ctypes.POINTER(ctypes.c_void_p)), recv_rows)
+    return _lib().moe_ep_attach(ctx, ctypes.byref(group), ctypes.c_void_p(cuda_stream))
+
+
+def moe_ep_route(ctx, logits_ptr: int, T: int, out: moe_dispatch_out, cuda_stream: int = 0) -> int:
+    return _lib().moe_ep_route(ctx, ctypes.c_void_p(logits_ptr), T, ctypes.byref(out),
+                               ctypes.c_void_p(cuda_stream))
+
+
+def moe_ep_scatter(ctx, x_ptr: int, T: int, counts_all_ptr: int, recv_slot_offsets_ptr: int,
+                   cuda_stream: int = 0) -> int:
+    vp = ctypes.c_void_p
+    return _lib().moe_ep_scatter(ctx, vp(x_ptr), T, vp(counts_all_ptr), vp(recv_slot_offsets_ptr),
+                                 vp(cuda_stream))
+
+
+def moe_ep_combine(ctx, T: int, y_ptr: int, cuda_stream: int = 0) -> int:
+    return _lib().moe_ep_combine(ctx, T, ctypes.c_void_p(y_ptr), ctypes.c_void_p(cuda_stream))
+
+
+def moe_ep_plan_host(counts_all, rank: int):
+    """Host-only layout of the exchange.  counts_all: [world, P] ints.
+    Returns (status, src_base i32[P], recv_slot_offsets i32[P/world + 1])."""
+    c = _i32(counts_all)
+    world, P = c.shape
+    src_base = np.zeros(P, np.int32)
+    recv_off = np.zeros(P // max(world, 1) + 1, np.int32)
+    st = _lib().moe_ep_plan_host(_np_ptr(c), world, rank, P, _np_ptr(src_base), _np_ptr(recv_off))
+    return st, src_base, recv_off
+
+
 def moe_route_destroy(ctx) -> int:
     return _lib().moe_route_destroy(ctx)
 
@@ -357,6 +407,38 @@ class MoeRouter:
         st = moe_combine(self._ctx, expert_buf.data_ptr(), T, y.data_ptr(), self._stream())
         if st != MOE_OK:
             raise MoeError(st, "moe_combine")
+        return y
+
+    # -- expert parallelism over several GPUs -------------------------------
+    def ep_attach(self, world: int, rank: int, recv_buf_ptrs, recv_rows: int) -> None:
+        st = moe_ep_attach(self._ctx, world, rank, recv_buf_ptrs, recv_rows, self._stream())
+        if st != MOE_OK:
+            raise MoeError(st, "moe_ep_attach")
+
+    def ep_route(self, logits: torch.Tensor, out: DispatchBuffers) -> DispatchBuffers:
+        T = logits.shape[0]
+        assert logits.dtype == torch.float32 and logits.is_contiguous() and logits.shape[1] == self.cfg.num_experts
+        st = moe_ep_route(self._ctx, logits.data_ptr(), T, out.as_struct(), self._stream())
+        if st != MOE_OK:
+            raise MoeError(st, "moe_ep_route")
+        return out
+
+    def ep_scatter(self, x: torch.Tensor, counts_all: torch.Tensor, recv_slot_offsets: torch.Tensor) -> None:
+        T = x.shape[0]
+        assert x.dtype == torch.bfloat16 and x.is_contiguous() and x.shape[1] == self.cfg.hidden
+        assert counts_all.dtype == torch.int32 and counts_all.is_contiguous()
+        assert recv_slot_offsets.dtype == torch.int32 and recv_slot_offsets.is_contiguous()
+        st = moe_ep_scatter(self._ctx, x.data_ptr(), T, counts_all.data_ptr(),
+                            recv_slot_offsets.data_ptr(), self._stream())
+        if st != MOE_OK:
+            raise MoeError(st, "moe_ep_scatter")
+
+    def ep_combine(self, T: int, y: torch.Tensor | None = None) -> torch.Tensor:
+        if y is None:
+            y = torch.empty((T, self.cfg.hidden), dtype=torch.bfloat16, device=self.device)
+        st = moe_ep_combine(self._ctx, T, y.data_ptr(), self._stream())
+        if st != MOE_OK:
+            raise MoeError(st, "moe_ep_combine")
         return y
 
     def step_host(self, logits_host: torch.Tensor, x_host: torch.Tensor, out: DispatchBuffers,

@@ -9,7 +9,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(CSRC, "libmoe_route.so")
 SOURCES = ["moe_route.cu", "permute_static.cu"]
-HEADERS = ["device_utils.cuh", "route_kernels.cuh", "scatter_kernels.cuh", "combine_kernels.cuh",
+HEADERS = ["device_utils.cuh", "route_kernels.cuh", "scatter_kernels.cuh", "combine_kernels.cuh", "ep_kernels.cuh",
            os.path.join("..", "..", "include", "moe_route.h")]
 
 

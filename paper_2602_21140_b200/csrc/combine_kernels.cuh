@@ -19,6 +19,11 @@ struct CombineParams {
     const float *topk_weights;   // [T,k]
     const int32_t *topk_slot;    // [T,k]
     const float *slot_scale;     // [P]
+    // Expert parallelism over several GPUs: the rows of slot p live in the receive buffer of
+    // GPU p / slots_per_gpu, reached through peer_bufs[that GPU]; dst_row then counts rows of
+    // that buffer.  NULL = every row is in `buf`.
+    const uint4 *const *peer_bufs;
+    int slots_per_gpu;
 };
 
 constexpr int kCombineThreads = 256;
@@ -120,18 +125,20 @@ constexpr int kCombineBulkMaxWarps = 8;   // warps per CTA (blockDim.x / 32), ea
 
 struct CombineIssue {   // per-lane state of the issuing side (lane j < k)
     int token;
-    int row, row_next;
+    const uint4 *row, *row_next;   // first 16-byte unit of the lane's source row
     float coef, coef_next;
 };
 
-__device__ __forceinline__ void combine_fetch_index(const CombineParams &p, int t, int lane, int &row,
-                                                    float &coef)
+__device__ __forceinline__ void combine_fetch_index(const CombineParams &p, int t, int lane,
+                                                    const uint4 *&row, float &coef)
 {
-    row = 0; coef = 0.0f;
+    row = p.buf; coef = 0.0f;
     if (lane < p.k && t < p.T) {
         const size_t i = (size_t)t * p.k + lane;
-        row = __ldg(p.dst_row + i);
-        coef = __fmul_rn(__ldg(p.topk_weights + i), __ldg(p.slot_scale + __ldg(p.topk_slot + i)));
+        const int slot = __ldg(p.topk_slot + i);
+        const uint4 *base = p.peer_bufs ? p.peer_bufs[slot / p.slots_per_gpu] : p.buf;
+        row = base + (size_t)__ldg(p.dst_row + i) * p.hv;
+        coef = __fmul_rn(__ldg(p.topk_weights + i), __ldg(p.slot_scale + slot));
     }
 }
 
@@ -192,7 +199,7 @@ __global__ void __launch_bounds__(kCombineBulkMaxWarps * 32) k_combine_bulk(Comb
         if (lane < k) {
             coefs[s * k + lane] = is.coef;
             bulk_load(ring + (size_t)s * stage_bytes + (size_t)lane * kChunkBytes,
-                      p.buf + (size_t)is.row * p.hv + c0, bytes, &full[s]);
+                      is.row + c0, bytes, &full[s]);
         }
     };
 

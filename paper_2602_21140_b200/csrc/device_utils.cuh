@@ -9,6 +9,7 @@ namespace moe {
 // Values of the device status word (mirrors moe_status where it applies).
 constexpr int kDevOk = 0;
 constexpr int kDevInsufficientExperts = 3;   // a token met fewer than k selectable experts
+constexpr int kDevCapacity = 4;              // rows of an exchange did not fit the receive buffer
 constexpr int kDevTimeout = 5;               // a bounded wait gave up
 
 // Bounded waits: polls before a waiter gives up, and the back-off between polls.

@@ -13,6 +13,7 @@
 #include <vector>
 
 #include "combine_kernels.cuh"
+#include "ep_kernels.cuh"
 #include "route_kernels.cuh"
 #include "scatter_kernels.cuh"
 
@@ -234,6 +235,12 @@ struct moe_ctx {
     const int32_t *last_dst_row;
     int32_t last_T;
     cudaEvent_t timing_event;   // optional: recorded between routing and scatter
+    // expert parallelism over several GPUs (moe_ep_attach)
+    int ep_world, ep_rank, ep_spg;
+    long long ep_recv_rows;
+    uint4 **d_peer_bufs;        // device [ep_world]
+    int32_t *d_src_base;        // device [P]
+    bool ep_routed;             // the latest routing came from moe_ep_route
 };
 
 namespace {
@@ -318,6 +325,45 @@ cudaError_t launch_combine(const CombineParams &p, int blocks, cudaStream_t st)
     return cudaGetLastError();
 }
 
+// The routing kernel of a dispatch (a1..a9 except the final row addition).
+cudaError_t enqueue_route(moe_ctx *ctx, const float *logits, int32_t T, const moe_dispatch_out *out,
+                          cudaStream_t st)
+{
+    const Derived &d = ctx->d;
+    RouteParams rp;
+    rp.logits = logits; rp.T = T; rp.E = d.E; rp.k = d.k; rp.P = d.P; rp.R = d.R; rp.S = d.S;
+    rp.max_rep = d.max_rep; rp.score_func = ctx->cfg.score_func; rp.n_group = ctx->cfg.n_group;
+    rp.topk_group = ctx->cfg.topk_group; rp.lanes_per_group = d.lanes_per_group;
+    rp.group_m = d.group_m; rp.route_scale = ctx->cfg.route_scale;
+    rp.tokens_per_block = d.tokens_per_block; rp.rank_words = d.rank_words;
+    rp.expert_words = d.expert_words;
+    rp.state = ctx->d_state; rp.bias = ctx->d_bias;
+    rp.topk_ids = out->topk_ids; rp.topk_weights = out->topk_weights; rp.topk_slot = out->topk_slot;
+    rp.pos_in_slot = ctx->d_pos;
+    rp.slot_counts = out->slot_counts; rp.slot_offsets = out->slot_offsets;
+    rp.rank_counts = out->rank_counts; rp.rank_offsets = out->rank_offsets;
+    rp.desc = ctx->d_desc; rp.ctl = ctx->d_ctl;
+    const int tiles = (T + d.tokens_per_block - 1) / d.tokens_per_block;
+    return launch_route(d.epl, d.lpt, rp, tiles, ctx->route_smem, st, ctx->pdl);
+}
+
+// The bulk-copy ring combine over `cp` (rows in one buffer, or in the peers' receive buffers).
+moe_status enqueue_combine_bulk(moe_ctx *ctx, const CombineParams &cp, cudaStream_t st)
+{
+    const int chunk_v = 32 * ctx->combine_u;
+    const long long items = (long long)cp.T * ((cp.hv + chunk_v - 1) / chunk_v);
+    const int nw = ctx->combine_warps;
+    const long long want = (items + nw - 1) / nw;
+    const int grid = (int)std::min<long long>(want, (long long)ctx->sm_count * ctx->combine_ctas_per_sm);
+    if (ctx->combine_u == 1)
+        launch_kernel(k_combine_bulk<1>, dim3(grid), dim3(nw * 32), ctx->combine_smem, st, ctx->pdl, cp, ctx->combine_stages, ctx->d_ctl);
+    else if (ctx->combine_u == 2)
+        launch_kernel(k_combine_bulk<2>, dim3(grid), dim3(nw * 32), ctx->combine_smem, st, ctx->pdl, cp, ctx->combine_stages, ctx->d_ctl);
+    else
+        launch_kernel(k_combine_bulk<4>, dim3(grid), dim3(nw * 32), ctx->combine_smem, st, ctx->pdl, cp, ctx->combine_stages, ctx->d_ctl);
+    return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Copy `words` leading words of `blob` to the device state through a pinned
@@ -349,6 +395,7 @@ void free_ctx(moe_ctx *ctx)
     if (!ctx) return;
     cudaFree(ctx->d_state); cudaFree(ctx->d_bias); cudaFree(ctx->d_slot_scale);
     cudaFree(ctx->d_desc); cudaFree(ctx->d_ctl); cudaFree(ctx->d_pos);
+    cudaFree(ctx->d_peer_bufs); cudaFree(ctx->d_src_base);
     for (int s = 0; s < kStagingSlots; ++s) {
         if (ctx->h_stage[s]) cudaFreeHost(ctx->h_stage[s]);
         if (ctx->stage_done[s]) cudaEventDestroy(ctx->stage_done[s]);
@@ -433,6 +480,8 @@ moe_status moe_route_init(const moe_config *cfg, const int32_t *slot_to_expert, 
     ctx->last_weights = nullptr; ctx->last_slot = nullptr; ctx->last_dst_row = nullptr;
     ctx->last_T = -1;
     ctx->timing_event = nullptr;
+    ctx->ep_world = 0; ctx->ep_rank = 0; ctx->ep_spg = 0; ctx->ep_recv_rows = 0;
+    ctx->d_peer_bufs = nullptr; ctx->d_src_base = nullptr; ctx->ep_routed = false;
     ctx->stage_next = 0;
     for (int s = 0; s < kStagingSlots; ++s) {
         ctx->h_stage[s] = nullptr; ctx->stage_done[s] = nullptr; ctx->stage_used[s] = false;
@@ -663,21 +712,8 @@ moe_status moe_dispatch(moe_ctx *ctx, const float *logits, const void *x, int32_
     ctx->last_weights = out->topk_weights; ctx->last_slot = out->topk_slot;
     ctx->last_dst_row = out->dst_row; ctx->last_T = T;
 
-    RouteParams rp;
-    rp.logits = logits; rp.T = T; rp.E = d.E; rp.k = d.k; rp.P = d.P; rp.R = d.R; rp.S = d.S;
-    rp.max_rep = d.max_rep; rp.score_func = ctx->cfg.score_func; rp.n_group = ctx->cfg.n_group;
-    rp.topk_group = ctx->cfg.topk_group; rp.lanes_per_group = d.lanes_per_group;
-    rp.group_m = d.group_m; rp.route_scale = ctx->cfg.route_scale;
-    rp.tokens_per_block = d.tokens_per_block; rp.rank_words = d.rank_words;
-    rp.expert_words = d.expert_words;
-    rp.state = ctx->d_state; rp.bias = ctx->d_bias;
-    rp.topk_ids = out->topk_ids; rp.topk_weights = out->topk_weights; rp.topk_slot = out->topk_slot;
-    rp.pos_in_slot = ctx->d_pos;
-    rp.slot_counts = out->slot_counts; rp.slot_offsets = out->slot_offsets;
-    rp.rank_counts = out->rank_counts; rp.rank_offsets = out->rank_offsets;
-    rp.desc = ctx->d_desc; rp.ctl = ctx->d_ctl;
-    const int tiles = (T + d.tokens_per_block - 1) / d.tokens_per_block;
-    if (launch_route(d.epl, d.lpt, rp, tiles, ctx->route_smem, st, ctx->pdl) != cudaSuccess) return MOE_ERR_CUDA;
+    if (enqueue_route(ctx, logits, T, out, st) != cudaSuccess) return MOE_ERR_CUDA;
+    ctx->ep_routed = false;
     if (ctx->timing_event && cudaEventRecord(ctx->timing_event, st) != cudaSuccess) return MOE_ERR_CUDA;
 
     ScatterParams sp;
@@ -711,7 +747,7 @@ moe_status moe_dispatch(moe_ctx *ctx, const float *logits, const void *x, int32_
 moe_status moe_combine(moe_ctx *ctx, const void *expert_buf, int32_t T, void *y, void *cuda_stream)
 {
     if (!ctx || T < 0) return MOE_ERR_INVALID_ARG;
-    if (ctx->last_T < 0 || T != ctx->last_T) return MOE_ERR_INVALID_ARG;
+    if (ctx->last_T < 0 || T != ctx->last_T || ctx->ep_routed) return MOE_ERR_INVALID_ARG;
     if (T == 0) return MOE_OK;
     if (!expert_buf || !y || !aligned16(expert_buf) || !aligned16(y)) return MOE_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -721,26 +757,153 @@ moe_status moe_combine(moe_ctx *ctx, const void *expert_buf, int32_t T, void *y,
     cp.T = T; cp.k = d.k; cp.hv = d.H / 8;
     cp.dst_row = ctx->last_dst_row; cp.topk_weights = ctx->last_weights; cp.topk_slot = ctx->last_slot;
     cp.slot_scale = ctx->d_slot_scale;
-    if (ctx->combine_impl == 1) {
-        const int chunk_v = 32 * ctx->combine_u;
-        const long long items = (long long)T * ((cp.hv + chunk_v - 1) / chunk_v);
-        const int nw = ctx->combine_warps;
-        const long long want = (items + nw - 1) / nw;
-        const int grid = (int)std::min<long long>(want, (long long)ctx->sm_count * ctx->combine_ctas_per_sm);
-        if (ctx->combine_u == 1)
-            launch_kernel(k_combine_bulk<1>, dim3(grid), dim3(nw * 32), ctx->combine_smem, st, ctx->pdl, cp, ctx->combine_stages, ctx->d_ctl);
-        else if (ctx->combine_u == 2)
-            launch_kernel(k_combine_bulk<2>, dim3(grid), dim3(nw * 32), ctx->combine_smem, st, ctx->pdl, cp, ctx->combine_stages, ctx->d_ctl);
-        else
-            launch_kernel(k_combine_bulk<4>, dim3(grid), dim3(nw * 32), ctx->combine_smem, st, ctx->pdl, cp, ctx->combine_stages, ctx->d_ctl);
-        return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
-    }
+    cp.peer_bufs = nullptr; cp.slots_per_gpu = 0;
+    if (ctx->combine_impl == 1) return enqueue_combine_bulk(ctx, cp, st);
     const int chunks = (cp.hv + kCombineChunk - 1) / kCombineChunk;
     const long long items = (long long)T * chunks;
     const long long want = (items + kCombineThreads / 32 - 1) / (kCombineThreads / 32);
     const int grid = (int)std::min<long long>(want, (long long)ctx->sm_count * ctx->combine_blocks_per_sm);
     if (launch_combine(cp, grid, st) != cudaSuccess) return MOE_ERR_CUDA;
     return MOE_OK;
+}
+
+// ---------------------------------------------------------------------------
+// Expert parallelism over several GPUs
+// ---------------------------------------------------------------------------
+
+moe_status moe_ep_plan_host(const int32_t *counts_all, int32_t world, int32_t rank, int32_t num_slots,
+                            int32_t *src_base, int32_t *recv_slot_offsets)
+{
+    if (!counts_all || world < 1 || rank < 0 || rank >= world || num_slots < 1 || num_slots % world != 0)
+        return MOE_ERR_INVALID_ARG;
+    const int spg = num_slots / world;
+    for (int s = 0; s < num_slots && src_base; ++s) {
+        const int first = (s / spg) * spg;
+        long long base = 0;
+        for (int q = first; q < s; ++q)
+            for (int g = 0; g < world; ++g) base += counts_all[(size_t)g * num_slots + q];
+        for (int g = 0; g < rank; ++g) base += counts_all[(size_t)g * num_slots + s];
+        if (base > 0x7fffffffll) return MOE_ERR_CAPACITY;
+        src_base[s] = (int32_t)base;
+    }
+    long long off = 0;
+    for (int q = 0; q <= spg && recv_slot_offsets; ++q) {
+        if (off > 0x7fffffffll) return MOE_ERR_CAPACITY;
+        recv_slot_offsets[q] = (int32_t)off;
+        if (q < spg)
+            for (int g = 0; g < world; ++g) off += counts_all[(size_t)g * num_slots + (size_t)rank * spg + q];
+    }
+    return MOE_OK;
+}
+
+moe_status moe_ep_attach(moe_ctx *ctx, const moe_ep_group *group, void *cuda_stream)
+{
+    if (!ctx || !group || !group->recv_bufs) return MOE_ERR_INVALID_ARG;
+    const Derived &d = ctx->d;
+    if (group->world < 1 || group->world > 1024 || group->rank < 0 || group->rank >= group->world)
+        return MOE_ERR_INVALID_ARG;
+    if (d.R % group->world != 0) return MOE_ERR_INVALID_ARG;          // whole simulated ranks per GPU
+    if (group->recv_rows < 1 || group->recv_rows > 0x7fffffffll) return MOE_ERR_INVALID_ARG;
+    if (ctx->combine_impl != 1) return MOE_ERR_INVALID_ARG;           // the ring combine is the peer-aware one
+    for (int r = 0; r < d.R; ++r)                                     // physical rank numbering only
+        if (ctx->n_listed != d.R || ctx->rank_order[r] != r) return MOE_ERR_INVALID_ARG;
+    for (int g = 0; g < group->world; ++g)
+        if (!group->recv_bufs[g] || !aligned16(group->recv_bufs[g])) return MOE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (stream_is_capturing(st)) return MOE_ERR_INVALID_ARG;
+    if (ctx->ep_world != group->world) {
+        cudaFree(ctx->d_peer_bufs); ctx->d_peer_bufs = nullptr; ctx->ep_world = 0;
+        if (cudaMalloc(&ctx->d_peer_bufs, (size_t)group->world * sizeof(uint4 *)) != cudaSuccess) {
+            cudaGetLastError();
+            return MOE_ERR_CUDA;
+        }
+    }
+    if (!ctx->d_src_base && cudaMalloc(&ctx->d_src_base, (size_t)d.P * 4) != cudaSuccess) {
+        cudaGetLastError();
+        return MOE_ERR_CUDA;
+    }
+    // synchronous copy: the host array may be freed on return
+    if (cudaMemcpyAsync(ctx->d_peer_bufs, group->recv_bufs, (size_t)group->world * sizeof(void *),
+                        cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess)
+        return MOE_ERR_CUDA;
+    ctx->ep_world = group->world; ctx->ep_rank = group->rank; ctx->ep_spg = d.P / group->world;
+    ctx->ep_recv_rows = group->recv_rows;
+    return MOE_OK;
+}
+
+moe_status moe_ep_route(moe_ctx *ctx, const float *logits, int32_t T, const moe_dispatch_out *out,
+                        void *cuda_stream)
+{
+    if (!ctx || !out || T < 0) return MOE_ERR_INVALID_ARG;
+    if (ctx->ep_world < 1) return MOE_ERR_INVALID_ARG;
+    if (T > ctx->cfg.max_tokens) return MOE_ERR_CAPACITY;
+    if (!out->slot_counts) return MOE_ERR_INVALID_ARG;
+    if (T > 0 && (!out->topk_ids || !out->topk_weights || !out->topk_slot || !out->slot_offsets ||
+                  !out->rank_counts || !out->rank_offsets || !out->dst_row))
+        return MOE_ERR_INVALID_ARG;
+    if (T > 0 && ((!logits && ctx->cfg.score_func != MOE_ROUTE_DENSE_TP) || !aligned16(logits)))
+        return MOE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    ctx->last_weights = out->topk_weights; ctx->last_slot = out->topk_slot;
+    ctx->last_dst_row = out->dst_row; ctx->last_T = T; ctx->ep_routed = true;
+    if (T == 0) {                      // this GPU sends nothing, but its counts still take part in the exchange
+        if (cudaMemsetAsync(out->slot_counts, 0, (size_t)ctx->d.P * 4, st) != cudaSuccess) return MOE_ERR_CUDA;
+        return MOE_OK;
+    }
+    return enqueue_route(ctx, logits, T, out, st) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+moe_status moe_ep_scatter(moe_ctx *ctx, const void *x, int32_t T, const int32_t *counts_all,
+                          int32_t *recv_slot_offsets, void *cuda_stream)
+{
+    if (!ctx || T < 0 || !counts_all || !recv_slot_offsets) return MOE_ERR_INVALID_ARG;
+    if (ctx->ep_world < 1 || !ctx->ep_routed || T != ctx->last_T) return MOE_ERR_INVALID_ARG;
+    if (T > 0 && (!x || !aligned16(x))) return MOE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const Derived &d = ctx->d;
+    EpPlanParams pp;
+    pp.counts = counts_all; pp.G = ctx->ep_world; pp.g = ctx->ep_rank; pp.P = d.P; pp.spg = ctx->ep_spg;
+    pp.recv_rows = ctx->ep_recv_rows; pp.src_base = ctx->d_src_base;
+    pp.recv_slot_offsets = recv_slot_offsets; pp.ctl = ctx->d_ctl;
+    if (launch_kernel(k_ep_plan, dim3(1), dim3(kEpPlanThreads), 0, st, false, pp) != cudaSuccess)
+        return MOE_ERR_CUDA;
+    if (T == 0) return MOE_OK;
+    EpScatterParams sp;
+    sp.x = static_cast<const uint4 *>(x); sp.peer_bufs = ctx->d_peer_bufs;
+    sp.T = T; sp.k = d.k; sp.hv = d.H / 8; sp.spg = ctx->ep_spg; sp.recv_rows = ctx->ep_recv_rows;
+    sp.topk_slot = ctx->last_slot; sp.src_base = ctx->d_src_base; sp.pos_in_slot = ctx->d_pos;
+    sp.dst_row = const_cast<int32_t *>(ctx->last_dst_row);
+    const int un = ctx->scatter_unroll;
+    const int chunks = (sp.hv + 32 * un - 1) / (32 * un);
+    const long long items = (long long)T * chunks;
+    const long long want = (items + kEpScatterThreads / 32 - 1) / (kEpScatterThreads / 32);
+    const int grid = (int)std::min<long long>(want, (long long)ctx->sm_count * ctx->scatter_blocks_per_sm);
+    switch (un) {
+        case 8: launch_kernel(k_ep_scatter<8>, dim3(grid), dim3(kEpScatterThreads), 0, st, ctx->pdl, sp); break;
+        case 16: launch_kernel(k_ep_scatter<16>, dim3(grid), dim3(kEpScatterThreads), 0, st, ctx->pdl, sp); break;
+        case 28: launch_kernel(k_ep_scatter<28>, dim3(grid), dim3(kEpScatterThreads), 0, st, ctx->pdl, sp); break;
+        case 32: launch_kernel(k_ep_scatter<32>, dim3(grid), dim3(kEpScatterThreads), 0, st, ctx->pdl, sp); break;
+        default: launch_kernel(k_ep_scatter<4>, dim3(grid), dim3(kEpScatterThreads), 0, st, ctx->pdl, sp); break;
+    }
+    return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+moe_status moe_ep_combine(moe_ctx *ctx, int32_t T, void *y, void *cuda_stream)
+{
+    if (!ctx || T < 0) return MOE_ERR_INVALID_ARG;
+    if (ctx->ep_world < 1 || !ctx->ep_routed || T != ctx->last_T) return MOE_ERR_INVALID_ARG;
+    if (T == 0) return MOE_OK;
+    if (!y || !aligned16(y)) return MOE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const Derived &d = ctx->d;
+    CombineParams cp;
+    cp.buf = nullptr; cp.y = static_cast<uint4 *>(y);
+    cp.T = T; cp.k = d.k; cp.hv = d.H / 8;
+    cp.dst_row = ctx->last_dst_row; cp.topk_weights = ctx->last_weights; cp.topk_slot = ctx->last_slot;
+    cp.slot_scale = ctx->d_slot_scale;
+    cp.peer_bufs = const_cast<const uint4 *const *>(ctx->d_peer_bufs); cp.slots_per_gpu = ctx->ep_spg;
+    return enqueue_combine_bulk(ctx, cp, st);
 }
 
 moe_status moe_step_host(moe_ctx *ctx, const float *logits_host, const void *x_host, int32_t T,
