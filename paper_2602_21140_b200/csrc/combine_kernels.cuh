@@ -123,12 +123,6 @@ __global__ void __launch_bounds__(kCombineThreads) k_combine_vec(CombineParams p
 // are fetched one token ahead.
 constexpr int kCombineBulkMaxWarps = 8;   // warps per CTA (blockDim.x / 32), each with its own ring
 
-struct CombineIssue {   // per-lane state of the issuing side (lane j < k)
-    int token;
-    const uint4 *row, *row_next;   // first 16-byte unit of the lane's source row
-    float coef, coef_next;
-};
-
 __device__ __forceinline__ void combine_fetch_index(const CombineParams &p, int t, int lane,
                                                     const uint4 *&row, float &coef)
 {
@@ -142,7 +136,10 @@ __device__ __forceinline__ void combine_fetch_index(const CombineParams &p, int 
     }
 }
 
-template <int U>
+// U = 16-byte units per lane and row chunk; K > 0: top_k known at compile time (the row loop
+// is unrolled), K == 0: any top_k.  All item bookkeeping is incremental: the loop is close to
+// being bound by instruction issue, so no division or modulo runs per item.
+template <int U, int K>
 __global__ void __launch_bounds__(kCombineBulkMaxWarps * 32) k_combine_bulk(CombineParams p, int stages,
                                                                          Control *ctl)
 {
@@ -151,7 +148,7 @@ __global__ void __launch_bounds__(kCombineBulkMaxWarps * 32) k_combine_bulk(Comb
     constexpr unsigned kChunkBytes = kChunkV * 16u;
     const int lane = lane_id(), warp = threadIdx.x >> 5;
     const int kCombineBulkWarps = blockDim.x >> 5;
-    const int k = p.k;
+    const int k = (K > 0) ? K : p.k;
     const unsigned stage_bytes = (unsigned)k * kChunkBytes;
     // per-warp carve-up: [stages][k][chunk] data, then [stages][k] coefficients, then barriers
     const size_t warp_bytes = (size_t)stages * stage_bytes;
@@ -179,65 +176,85 @@ __global__ void __launch_bounds__(kCombineBulkMaxWarps * 32) k_combine_bulk(Comb
     const int n_mine = (int)(per + (wid < extra ? 1 : 0));
     if (n_mine == 0) return;
 
-    CombineIssue is;
-    is.token = (int)(first / chunks);
-    combine_fetch_index(p, is.token, lane, is.row, is.coef);
-    combine_fetch_index(p, is.token + 1, lane, is.row_next, is.coef_next);
+    // issuing side: token / chunk / stage of the next item to request (lane j < k owns row j)
+    int it_tok = (int)(first / chunks), it_chunk = (int)(first % chunks), it_stage = 0;
+    const uint4 *row, *row_next; float coef, coef_next;
+    combine_fetch_index(p, it_tok, lane, row, coef);
+    combine_fetch_index(p, it_tok + 1, lane, row_next, coef_next);
 
-    auto issue = [&](int n) {
-        const long long item = first + n;
-        const int t = (int)(item / chunks);
-        const int c0 = (int)(item % chunks) * kChunkV;
-        if (t != is.token) {                               // moved on: take the prefetched indices
-            is.token = t; is.row = is.row_next; is.coef = is.coef_next;
-            combine_fetch_index(p, t + 1, lane, is.row_next, is.coef_next);
-        }
-        const int s = n % stages;
+    auto issue = [&]() {
+        const int c0 = it_chunk * kChunkV;
         const unsigned bytes = (unsigned)min(kChunkV, p.hv - c0) * 16u;
-        if (lane == 0) mbar_expect_tx(&full[s], bytes * (unsigned)k);
+        if (lane == 0) mbar_expect_tx(&full[it_stage], bytes * (unsigned)k);
         __syncwarp();
         if (lane < k) {
-            coefs[s * k + lane] = is.coef;
-            bulk_load(ring + (size_t)s * stage_bytes + (size_t)lane * kChunkBytes,
-                      is.row + c0, bytes, &full[s]);
+            coefs[it_stage * k + lane] = coef;
+            bulk_load(ring + (size_t)it_stage * stage_bytes + (size_t)lane * kChunkBytes, row + c0, bytes,
+                      &full[it_stage]);
+        }
+        if (++it_stage == stages) it_stage = 0;
+        if (++it_chunk == chunks) {                        // next token: take the prefetched indices
+            it_chunk = 0; ++it_tok;
+            row = row_next; coef = coef_next;
+            combine_fetch_index(p, it_tok + 1, lane, row_next, coef_next);
         }
     };
 
-    for (int n = 0; n < min(stages - 1, n_mine); ++n) issue(n);
+    const int ahead = min(stages - 1, n_mine);
+    for (int n = 0; n < ahead; ++n) issue();
 
+    // consuming side
+    int tok = (int)(first / chunks), chunk = (int)(first % chunks), stage = 0;
+    unsigned parity = 0;
     bool ok = true;
     int n = 0;
     for (; n < n_mine; ++n) {
-        if (n + stages - 1 < n_mine) issue(n + stages - 1);   // refills the stage consumed at n-1
-        const int s = n % stages;
-        const unsigned parity = (unsigned)(n / stages) & 1u;
+        if (n + stages - 1 < n_mine) issue();              // refills the stage consumed at n-1
         unsigned spins = 0;
-        while (!mbar_try_wait(&full[s], parity)) {
+        while (!mbar_try_wait(&full[stage], parity)) {
             if (++spins > kSpinLimit) { ok = false; break; }
         }
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         __syncwarp();                                      // coefficients written at issue are visible
-        const long long item = first + n;
-        const int t = (int)(item / chunks);
-        const int c0 = (int)(item % chunks) * kChunkV + lane;
+        const int c0 = chunk * kChunkV + lane;
         float acc[U][8];
 #pragma unroll
         for (int u = 0; u < U; ++u)
 #pragma unroll
             for (int q = 0; q < 8; ++q) acc[u][q] = 0.0f;
-        const uint4 *st = reinterpret_cast<const uint4 *>(ring + (size_t)s * stage_bytes);
-        for (int j = 0; j < k; ++j) {
-            const float c = coefs[s * k + j];
+        const uint4 *st = reinterpret_cast<const uint4 *>(ring + (size_t)stage * stage_bytes);
+        const float *cf = coefs + stage * k;
+        if (K > 0) {
+            uint4 v[K > 0 ? K : 1][U];
+            float c[K > 0 ? K : 1];
 #pragma unroll
-            for (int u = 0; u < U; ++u)
-                if (c0 + 32 * u < p.hv) fma_bf16x8(acc[u], st[j * kChunkV + lane + 32 * u], c);
+            for (int j = 0; j < K; ++j) {
+                c[j] = cf[j];
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+                    if (c0 + 32 * u < p.hv) v[j][u] = st[j * kChunkV + lane + 32 * u];
+            }
+#pragma unroll
+            for (int j = 0; j < K; ++j)
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+                    if (c0 + 32 * u < p.hv) fma_bf16x8(acc[u], v[j][u], c[j]);
+        } else {
+            for (int j = 0; j < k; ++j) {
+                const float c = cf[j];
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+                    if (c0 + 32 * u < p.hv) fma_bf16x8(acc[u], st[j * kChunkV + lane + 32 * u], c);
+            }
         }
-        uint4 *dst = p.y + (size_t)t * p.hv;
+        uint4 *dst = p.y + (size_t)tok * p.hv;
 #pragma unroll
         for (int u = 0; u < U; ++u)
             if (c0 + 32 * u < p.hv) st_stream_v4(dst + c0 + 32 * u, pack_bf16x8(acc[u]));
-        __syncwarp();                                      // every lane is done reading stage s
+        __syncwarp();                                      // every lane is done reading the stage
+        if (++stage == stages) { stage = 0; parity ^= 1u; }
+        if (++chunk == chunks) { chunk = 0; ++tok; }
     }
     if (!ok) {
         if (lane == 0) report_status(ctl, kDevTimeout);

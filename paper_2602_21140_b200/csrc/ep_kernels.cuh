@@ -26,22 +26,30 @@ struct EpPlanParams {
     Control *ctl;
 };
 
-// One small block; every output element is an independent plain sum over the table.
+// One small block.  First the total of every slot over all senders goes to shared memory,
+// then every output element is a plain sum over (part of) its owner's run of slots.
+constexpr int kEpMaxSlots = 4096;
+
 __global__ void __launch_bounds__(kEpPlanThreads) k_ep_plan(EpPlanParams p)
 {
+    __shared__ int32_t s_tot[kEpMaxSlots];
     pdl_enter();
+    for (int s = threadIdx.x; s < p.P; s += kEpPlanThreads) {
+        int tot = 0;
+        for (int g2 = 0; g2 < p.G; ++g2) tot += p.counts[(size_t)g2 * p.P + s];
+        s_tot[s] = tot;
+    }
+    __syncthreads();
     for (int s = threadIdx.x; s < p.P; s += kEpPlanThreads) {
         const int first = (s / p.spg) * p.spg;
         long long base = 0;
-        for (int q = first; q < s; ++q)
-            for (int g2 = 0; g2 < p.G; ++g2) base += p.counts[(size_t)g2 * p.P + q];
+        for (int q = first; q < s; ++q) base += s_tot[q];
         for (int g2 = 0; g2 < p.g; ++g2) base += p.counts[(size_t)g2 * p.P + s];
         p.src_base[s] = (int32_t)min(base, (long long)0x7fffffff);
     }
     for (int q = threadIdx.x; q <= p.spg; q += kEpPlanThreads) {
         long long off = 0;
-        for (int q2 = 0; q2 < q; ++q2)
-            for (int g2 = 0; g2 < p.G; ++g2) off += p.counts[(size_t)g2 * p.P + (size_t)p.g * p.spg + q2];
+        for (int q2 = 0; q2 < q; ++q2) off += s_tot[p.g * p.spg + q2];
         p.recv_slot_offsets[q] = (int32_t)min(off, (long long)0x7fffffff);
         if (q == p.spg && off > p.recv_rows) report_status(p.ctl, kDevCapacity);
     }
