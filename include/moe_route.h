@@ -308,6 +308,18 @@ moe_status moe_step_host(moe_ctx *ctx, const float *logits_host, const void *x_h
                          void *y_dev, void *y_host, void *cuda_stream);
 
 /*
+ * moe_step_host_async — moe_step_host without the final wait: everything, the copy of y
+ * to y_host included, is only enqueued on `cuda_stream`.  The host buffers must stay valid
+ * and y_host must not be read until the caller has synchronised with the stream.  With two
+ * contexts on two streams, each with its own staging and output buffers, the upload of one
+ * batch overlaps the download of the other (the link carries both directions at once),
+ * which is how micro-batches (Sec. 2.2) keep both directions busy.
+ */
+moe_status moe_step_host_async(moe_ctx *ctx, const float *logits_host, const void *x_host, int32_t T,
+                               const moe_dispatch_out *out, float *logits_dev, void *x_dev,
+                               void *y_dev, void *y_host, void *cuda_stream);
+
+/*
  * moe_set_timing_event — measurement hook (no counterpart in the paper).
  * `cuda_event` is a cudaEvent_t created by the caller with timing enabled, or
  * NULL to switch the hook off.  While set, every moe_dispatch records it on

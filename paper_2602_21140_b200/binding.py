@@ -37,7 +37,7 @@ MOE_ROUTE_DENSE_TP = 2
 
 EXPORTED_SYMBOLS = (
     "moe_route_init", "moe_set_failed_ranks", "moe_update_replica_map", "moe_dispatch",
-    "moe_combine", "moe_step_host", "moe_set_timing_event", "moe_get_device_status", "moe_plan_routing_state",
+    "moe_combine", "moe_step_host", "moe_step_host_async", "moe_set_timing_event", "moe_get_device_status", "moe_plan_routing_state",
     "moe_workspace_bytes", "moe_route_destroy", "moe_status_string", "moe_permute_static",
     "moe_set_failed_experts", "moe_compact_ranks", "moe_set_rank_order",
     "moe_ep_attach", "moe_ep_route", "moe_ep_scatter", "moe_ep_combine", "moe_ep_plan_host",
@@ -103,6 +103,8 @@ def _lib():
         lib.moe_combine.argtypes = [vp, vp, i32, vp, vp]
         lib.moe_step_host.restype = ctypes.c_int
         lib.moe_step_host.argtypes = [vp, vp, vp, i32, ctypes.POINTER(moe_dispatch_out), vp, vp, vp, vp, vp]
+        lib.moe_step_host_async.restype = ctypes.c_int
+        lib.moe_step_host_async.argtypes = [vp, vp, vp, i32, ctypes.POINTER(moe_dispatch_out), vp, vp, vp, vp, vp]
         lib.moe_set_timing_event.restype = ctypes.c_int
         lib.moe_set_timing_event.argtypes = [vp, vp]
         lib.moe_get_device_status.restype = ctypes.c_int
@@ -235,6 +237,15 @@ def moe_step_host(ctx, logits_host_ptr: int, x_host_ptr: int, T: int, out: moe_d
     return _lib().moe_step_host(ctx, vp(logits_host_ptr), vp(x_host_ptr), T, ctypes.byref(out),
                                 vp(logits_dev_ptr), vp(x_dev_ptr), vp(y_dev_ptr), vp(y_host_ptr),
                                 vp(cuda_stream))
+
+
+def moe_step_host_async(ctx, logits_host_ptr: int, x_host_ptr: int, T: int, out: moe_dispatch_out,
+                        logits_dev_ptr: int, x_dev_ptr: int, y_dev_ptr: int, y_host_ptr: int,
+                        cuda_stream: int = 0) -> int:
+    vp = ctypes.c_void_p
+    return _lib().moe_step_host_async(ctx, vp(logits_host_ptr), vp(x_host_ptr), T, ctypes.byref(out),
+                                      vp(logits_dev_ptr), vp(x_dev_ptr), vp(y_dev_ptr), vp(y_host_ptr),
+                                      vp(cuda_stream))
 
 
 def moe_set_timing_event(ctx, cuda_event: int) -> int:
@@ -450,6 +461,17 @@ class MoeRouter:
                            y_host.data_ptr(), self._stream())
         if st != MOE_OK:
             raise MoeError(st, "moe_step_host")
+
+    def step_host_async(self, logits_host: torch.Tensor, x_host: torch.Tensor, out: DispatchBuffers,
+                        logits_dev: torch.Tensor, x_dev: torch.Tensor, y_dev: torch.Tensor,
+                        y_host: torch.Tensor) -> None:
+        """As step_host, but returns once the work is enqueued on the current stream."""
+        T = logits_host.shape[0]
+        st = moe_step_host_async(self._ctx, logits_host.data_ptr(), x_host.data_ptr(), T, out.as_struct(),
+                                 logits_dev.data_ptr(), x_dev.data_ptr(), y_dev.data_ptr(),
+                                 y_host.data_ptr(), self._stream())
+        if st != MOE_OK:
+            raise MoeError(st, "moe_step_host_async")
 
     def set_timing_event(self, event: "torch.cuda.Event | None") -> None:
         """Record `event` between the routing and the scatter kernel of every dispatch."""

@@ -926,9 +926,9 @@ moe_status moe_ep_combine(moe_ctx *ctx, int32_t T, void *y, void *cuda_stream)
     return enqueue_combine_bulk(ctx, cp, st);
 }
 
-moe_status moe_step_host(moe_ctx *ctx, const float *logits_host, const void *x_host, int32_t T,
-                         const moe_dispatch_out *out, float *logits_dev, void *x_dev, void *y_dev,
-                         void *y_host, void *cuda_stream)
+moe_status moe_step_host_async(moe_ctx *ctx, const float *logits_host, const void *x_host, int32_t T,
+                               const moe_dispatch_out *out, float *logits_dev, void *x_dev, void *y_dev,
+                               void *y_host, void *cuda_stream)
 {
     if (!ctx || !out || T < 0) return MOE_ERR_INVALID_ARG;
     if (T > ctx->cfg.max_tokens) return MOE_ERR_CAPACITY;
@@ -947,8 +947,17 @@ moe_status moe_step_host(moe_ctx *ctx, const float *logits_host, const void *x_h
     if (ms != MOE_OK) return ms;
     if (T > 0 && cudaMemcpyAsync(y_host, y_dev, (size_t)T * d.H * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return MOE_ERR_CUDA;
-    if (cudaStreamSynchronize(st) != cudaSuccess) return MOE_ERR_CUDA;
     return MOE_OK;
+}
+
+moe_status moe_step_host(moe_ctx *ctx, const float *logits_host, const void *x_host, int32_t T,
+                         const moe_dispatch_out *out, float *logits_dev, void *x_dev, void *y_dev,
+                         void *y_host, void *cuda_stream)
+{
+    const moe_status ms = moe_step_host_async(ctx, logits_host, x_host, T, out, logits_dev, x_dev, y_dev,
+                                              y_host, cuda_stream);
+    if (ms != MOE_OK) return ms;
+    return cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
 moe_status moe_set_timing_event(moe_ctx *ctx, void *cuda_event)

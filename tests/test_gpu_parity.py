@@ -201,6 +201,40 @@ def test_step_from_host_memory():
     router.close()
 
 
+def test_two_host_fed_steps_in_flight():
+    # two contexts on two streams, nothing waited for until both steps are enqueued
+    wl = W.WORKLOADS["qwen3"]
+    T = 700
+    parts = []
+    for seed in (3, 4):
+        inp = W.make_inputs(wl, T=T, seed=seed)
+        router = make_router(wl, inp, max_tokens=T)
+        router.set_failed_ranks((5,))
+        parts.append(dict(
+            inp=inp, router=router, stream=torch.cuda.Stream(), out=router.alloc_outputs(T),
+            lg_h=torch.from_numpy(inp["logits"]).pin_memory(),
+            x_h=torch.from_numpy(inp["x"]).view(torch.int16).view(torch.bfloat16).pin_memory(),
+            y_h=torch.zeros((T, wl.H), dtype=torch.bfloat16).pin_memory(),
+            lg_d=torch.empty((T, wl.E), dtype=torch.float32, device="cuda"),
+            x_d=torch.empty((T, wl.H), dtype=torch.bfloat16, device="cuda"),
+            y_d=torch.empty((T, wl.H), dtype=torch.bfloat16, device="cuda")))
+    torch.cuda.synchronize()
+    for _ in range(3):
+        for p in parts:
+            with torch.cuda.stream(p["stream"]):
+                p["router"].step_host_async(p["lg_h"], p["x_h"], p["out"], p["lg_d"], p["x_d"], p["y_d"], p["y_h"])
+    for p in parts:
+        p["stream"].synchronize()
+        inp = p["inp"]
+        ref = oracle.dispatch(oracle_cfg(wl), inp["slot_to_expert"], (5,), None, inp["logits"], inp["x"])
+        check_dispatch(p["out"], ref)
+        ref_y = oracle.combine(ref["send_buf"], ref["dst_row"], ref["topk_weights"], ref["topk_slot"],
+                               inp["slot_scale"])
+        assert_y_close(p["y_h"].view(torch.int16).numpy().view(np.uint16), ref_y)
+        assert p["router"].device_status() == 0
+        p["router"].close()
+
+
 def test_argument_validation_on_device():
     wl = W.WORKLOADS["tiny"]
     inp = W.make_inputs(wl)
