@@ -16,18 +16,26 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "moe_oracle.c")
 _LIB = os.path.join(_HERE, "libmoe_oracle.so")
+# The mutation test points this front end at deliberately broken builds of the C source.
+_OVERRIDE = os.environ.get("MOE_ORACLE_LIB_OVERRIDE")
 _lib = None
+
+
+def compile_source(src: str, lib: str) -> None:
+    tmp = lib + f".tmp{os.getpid()}"
+    subprocess.check_call(
+        ["gcc", "-O2", "-ffp-contract=off", "-std=c11", "-Wall", "-shared", "-fPIC",
+         "-o", tmp, src, "-lm"])
+    os.replace(tmp, lib)
 
 
 def build(force: bool = False) -> str:
     """Compile the oracle with gcc (contraction off) if the library is stale."""
+    if _OVERRIDE:
+        return _OVERRIDE
     stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
     if force or stale:
-        tmp = _LIB + f".tmp{os.getpid()}"
-        subprocess.check_call(
-            ["gcc", "-O2", "-ffp-contract=off", "-std=c11", "-Wall", "-shared", "-fPIC",
-             "-o", tmp, _SRC, "-lm"])
-        os.replace(tmp, _LIB)
+        compile_source(_SRC, _LIB)
     return _LIB
 
 
@@ -61,8 +69,7 @@ class OracleConfig:
 def _load():
     global _lib
     if _lib is None:
-        build()
-        lib = ctypes.CDLL(_LIB)
+        lib = ctypes.CDLL(build())
         lib.oracle_exp_spec.restype = ctypes.c_float
         lib.oracle_exp_spec.argtypes = [ctypes.c_float]
         lib.oracle_sigmoid_spec.restype = ctypes.c_float
