@@ -60,7 +60,7 @@ struct RouteParams {
 __host__ __device__ inline size_t route_smem_bytes(int E, int max_rep, int tokens_per_block, int k,
                                                    int P)
 {
-    size_t words = (size_t)E + (size_t)E * max_rep + 2 * (size_t)tokens_per_block * k + 2 * (size_t)P;
+    size_t words = (size_t)E + (size_t)E * max_rep + 2 * (size_t)tokens_per_block * k + 3 * (size_t)P;
     return words * sizeof(int32_t) + (size_t)kRouteWarps * P * sizeof(uint16_t);
 }
 
@@ -243,7 +243,8 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
     int32_t *s_lrank = s_slot + NA;                   // [NA] stable rank inside the tile
     int32_t *s_hist = s_lrank + NA;                   // [P]  tile histogram (running)
     int32_t *s_excl = s_hist + P;                     // [P]  assignments on slot p in earlier tiles
-    uint16_t *s_wcount = reinterpret_cast<uint16_t *>(s_excl + P);   // [32][P] one round's counts
+    int32_t *s_order = s_excl + P;                    // [P]  physical slot at each layout position
+    uint16_t *s_wcount = reinterpret_cast<uint16_t *>(s_order + P);  // [32][P] one round's counts
     __shared__ unsigned s_ticket, s_epoch;
     __shared__ int s_warp_sums[kRouteWarps];
 
@@ -252,26 +253,38 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
 
     pdl_enter();
     if (tid == 0) {
-        s_epoch = ld_relaxed_u32(&p.ctl->epoch);
-        s_ticket = atomicAdd(&p.ctl->ticket, 1u);
+        // ticket (low word) and epoch (high word) share one 64-bit word: a single atomic add
+        // takes the ticket and reads the epoch (the ticket never carries: it is reset every step)
+        const unsigned long long te = atomicAdd(reinterpret_cast<unsigned long long *>(&p.ctl->ticket), 1ull);
+        s_ticket = (unsigned)te;
+        s_epoch = (unsigned)(te >> 32);
     }
     // Live replica lists from the rank bitmap and the replica table (a2, a6).
     const uint32_t *alive = reinterpret_cast<const uint32_t *>(p.state + kStateHeaderWords);
     const uint32_t *lost = alive + p.rank_words;
     const int32_t *table = p.state + kStateHeaderWords + p.rank_words + p.expert_words;
     for (int e = tid; e < E; e += kRouteThreads) {
+        // first every replica slot of the expert, then the alive words they point to: two
+        // rounds of independent loads instead of a chain through the replicas
+        constexpr int kMaxRep = 8;
+        int slot[kMaxRep];
+        uint32_t word[kMaxRep];
+        const uint32_t lost_word = lost[e >> 5];
+#pragma unroll
+        for (int r = 0; r < kMaxRep; ++r) slot[r] = (r < p.max_rep) ? table[e * p.max_rep + r] : -1;
+#pragma unroll
+        for (int r = 0; r < kMaxRep; ++r) word[r] = (slot[r] >= 0) ? alive[(slot[r] / p.S) >> 5] : 0u;
+        const bool expert_ok = !((lost_word >> (e & 31)) & 1u);
         int n = 0;
-        const bool expert_ok = !((lost[e >> 5] >> (e & 31)) & 1u);
-        for (int r = 0; r < p.max_rep && expert_ok; ++r) {
-            const int slot = table[e * p.max_rep + r];
-            if (slot >= 0) {
-                const int rank = slot / p.S;
-                if ((alive[rank >> 5] >> (rank & 31)) & 1u) s_live[e * p.max_rep + n++] = slot;
-            }
-        }
+#pragma unroll
+        for (int r = 0; r < kMaxRep; ++r)
+            if (expert_ok && slot[r] >= 0 && ((word[r] >> ((slot[r] / p.S) & 31)) & 1u))
+                s_live[e * p.max_rep + n++] = slot[r];
         s_nlive[e] = n;
     }
-    for (int q = tid; q < P; q += kRouteThreads) { s_hist[q] = 0; s_excl[q] = 0; }
+    // layout order of the slots, for the final scan of the last tile
+    const int32_t *order = p.state + kStateHeaderWords + p.rank_words + p.expert_words + E * p.max_rep;
+    for (int q = tid; q < P; q += kRouteThreads) { s_hist[q] = 0; s_excl[q] = 0; s_order[q] = order[q]; }
     for (int q = tid; q < kRouteWarps * P; q += kRouteThreads) s_wcount[q] = 0;
     const int fallback_expert = p.state[0];
     __syncthreads();
@@ -420,13 +433,12 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
     // ---- the last tile knows every total: a7 counts, a8 offsets -----------
     // exclusive scan over the P layout positions (position q holds physical slot order[q]),
     // a contiguous chunk of positions per thread
-    const int32_t *order = p.state + kStateHeaderWords + p.rank_words + p.expert_words + E * p.max_rep;
     for (int q = tid; q < P; q += kRouteThreads) s_hist[q] += s_excl[q];     // totals per physical slot
     __syncthreads();
     const int chunk = (P + kRouteThreads - 1) / kRouteThreads;
     const int q0 = tid * chunk;
     int local = 0;
-    for (int q = q0; q < min(P, q0 + chunk); ++q) local += s_hist[order[q]];
+    for (int q = q0; q < min(P, q0 + chunk); ++q) local += s_hist[s_order[q]];
     int incl = local;
     for (int off = 1; off < 32; off <<= 1) {
         const int o = __shfl_up_sync(full, incl, off);
@@ -438,7 +450,7 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
     for (int w2 = 0; w2 < warp; ++w2) warp_base += s_warp_sums[w2];
     int run = warp_base + incl - local;
     for (int q = q0; q < min(P, q0 + chunk); ++q) {
-        const int slot = order[q];
+        const int slot = s_order[q];
         const int tot = s_hist[slot];
         p.slot_counts[slot] = tot;
         p.slot_offsets[slot] = run;
@@ -452,7 +464,7 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
     __syncthreads();
     for (int r = tid; r < p.R; r += kRouteThreads) {   // r-th rank of the layout order
         int c = 0;
-        for (int s = 0; s < p.S; ++s) c += s_hist[order[r * p.S + s]];
+        for (int s = 0; s < p.S; ++s) c += s_hist[s_order[r * p.S + s]];
         p.rank_counts[r] = c;
         p.rank_offsets[r] = s_excl[r * p.S];
     }
