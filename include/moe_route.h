@@ -247,8 +247,8 @@ typedef struct {
 
 /*
  * moe_ep_attach — bind a context to its group: copies the pointer table to the device and
- * allocates the per-slot offset scratch (the only allocation of this mode; call it at
- * set-up, not while capturing).  May be called again with other buffers.
+ * allocates the per-slot offset scratch (the only allocation of this mode, 4*P + 8*world
+ * bytes on top of moe_workspace_bytes; call it at set-up, not while capturing).  May be called again with other buffers.
  * INVALID_ARG if num_ranks % world != 0, a pointer is NULL or misaligned, a rank order is
  * set, or the shape leaves no room for the bulk-copy combine.
  */
