@@ -152,3 +152,35 @@ def test_remap_while_capturing_is_refused():
         torch.zeros(1, device="cuda").add_(1)
     assert st == B.MOE_ERR_INVALID_ARG
     router.close()
+
+
+@pytest.mark.parametrize("name,T,replays", [("tiny", 128, 6000), ("dsv3", 2048, 1500)])
+def test_long_run_of_replays_with_remaps_stays_exact(name, T, replays):
+    # thousands of back-to-back replays of one graph, a remap every 37 steps: the look-back
+    # descriptors are recycled by their epoch tag and the ticket resets every step, so a rare
+    # ordering slip would show up as a changed result, a wrong total or a device status
+    wl = W.WORKLOADS[name]
+    inp = W.make_inputs(wl, T=T)
+    router = make_router(wl, inp, max_tokens=T)
+    logits, x = to_dev(inp["logits"]), to_dev(inp["x"], torch.bfloat16)      # the graph reads these: keep them
+    graph, out, y = _capture(router, logits, x, T)
+    sets = list(wl.failure_sets)
+    seen = {}
+    for i in range(replays):
+        if i % 37 == 0:
+            failed = sets[(i // 37) % len(sets)]
+            router.set_failed_ranks(failed)
+        graph.replay()
+        if i % 211 == 0 or i == replays - 1:
+            torch.cuda.synchronize()
+            assert int(out.slot_offsets[-1]) == T * wl.k
+            sig = (out.dst_row.clone(), y.clone())
+            if tuple(failed) in seen:
+                assert torch.equal(seen[tuple(failed)][0], sig[0]) and torch.equal(seen[tuple(failed)][1], sig[1])
+            seen.setdefault(tuple(failed), sig)
+    assert router.device_status() == 0
+    # and the result is the right one, not just a stable one
+    ref = _oracle_step(wl, inp, failed)
+    check_dispatch(out, ref)
+    assert_y_close(bf16_bits(y), ref["y"])
+    router.close()
