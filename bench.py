@@ -33,6 +33,7 @@ import numpy as np  # noqa: E402
 METRIC = "dispatch+combine tokens/s at DSv3 shape"
 UNIT = "tokens/s"
 N_INPUT_SETS = 3      # device copies of the inputs that the timed steps rotate over
+E2E_STEPS_IN_FLIGHT = int(os.environ.get("MOE_BENCH_E2E_IN_FLIGHT", "2"))   # host-fed steps kept in flight
 
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from ncu captures of
 # the kernels as they stand at the DSv3 shape (summaries under profiles/); None when a kernel
@@ -321,8 +322,8 @@ def run_ours(args):
                   "k_combine": statistics.mean(e[2].elapsed_time(e[3]) for e in ev)}
 
         # ---- end to end through the C ABI with host buffers ----------------
-        # Every step uploads its logits and x from pinned host memory and downloads its y.  Two
-        # steps are kept in flight (two contexts, two streams, separate staging and outputs), so
+        # Every step uploads its logits and x from pinned host memory and downloads its y.  A few
+        # steps are kept in flight (one context, stream, staging and output set each), so
         # that one step's upload overlaps the other's download; the one-at-a-time figure is
         # reported beside it.
         K3 = min(K, 20)
@@ -338,21 +339,22 @@ def run_ours(args):
         e2e_serial_s = max_over_ranks(time.perf_counter() - t0, world, dev)
         launches += 3 * (K3 + 2)
 
-        router2 = B.MoeRouter(B.config_for_workload(wl, max_tokens=T), inp["slot_to_expert"], bias,
-                              inp["slot_scale"], device=dev)
-        router2.set_failed_ranks(failed)
-        lanes = [dict(r=router, st=stream, out=out, lg_d=lg_d, x_d=x_d, y=y, y_h=y_h),
-                 dict(r=router2, st=torch.cuda.Stream(device=dev), out=router2.alloc_outputs(T),
-                      lg_d=torch.empty_like(logits), x_d=torch.empty_like(x), y=torch.empty_like(y),
-                      y_h=torch.empty((T, wl.H), dtype=torch.bfloat16).pin_memory())]
+        lanes = [dict(r=router, st=stream, out=out, lg_d=lg_d, x_d=x_d, y=y, y_h=y_h)]
+        for _ in range(E2E_STEPS_IN_FLIGHT - 1):
+            r_extra = B.MoeRouter(B.config_for_workload(wl, max_tokens=T), inp["slot_to_expert"], bias,
+                                  inp["slot_scale"], device=dev)
+            r_extra.set_failed_ranks(failed)
+            lanes.append(dict(r=r_extra, st=torch.cuda.Stream(device=dev), out=r_extra.alloc_outputs(T),
+                              lg_d=torch.empty_like(logits), x_d=torch.empty_like(x), y=torch.empty_like(y),
+                              y_h=torch.empty((T, wl.H), dtype=torch.bfloat16).pin_memory()))
 
         def host_step(i):
-            ln = lanes[i % 2]
+            ln = lanes[i % E2E_STEPS_IN_FLIGHT]
             ln["st"].synchronize()                       # the lane's previous step has delivered its y
             with torch.cuda.stream(ln["st"]):
                 ln["r"].step_host_async(lg_h, x_h, ln["out"], ln["lg_d"], ln["x_d"], ln["y"], ln["y_h"])
 
-        for i in range(4):
+        for i in range(2 * E2E_STEPS_IN_FLIGHT):
             host_step(i)
         torch.cuda.synchronize()
         if world > 1:
@@ -362,13 +364,14 @@ def run_ours(args):
             host_step(i)
         torch.cuda.synchronize()
         e2e_s = max_over_ranks(time.perf_counter() - t0, world, dev)
-        launches += 3 * (K3 + 4)
-        assert router2.device_status() == 0
-        assert torch.equal(lanes[0]["y_h"], lanes[1]["y_h"])          # both lanes computed the same batch
-        router2.close()
+        launches += 3 * (K3 + 2 * E2E_STEPS_IN_FLIGHT)
+        for ln in lanes[1:]:
+            assert ln["r"].device_status() == 0
+            assert torch.equal(lanes[0]["y_h"], ln["y_h"])            # every lane computed the same batch
+            ln["r"].close()
         e2e = {"value": world * T * K3 / e2e_s, "unit": UNIT,
                "h2d_bytes_per_step": T * wl.E * 4 + T * wl.H * 2, "d2h_bytes_per_step": T * wl.H * 2,
-               "steps": K3, "ms_per_step": 1e3 * e2e_s / K3, "steps_in_flight": 2,
+               "steps": K3, "ms_per_step": 1e3 * e2e_s / K3, "steps_in_flight": E2E_STEPS_IN_FLIGHT,
                "one_step_at_a_time": {"value": world * T * K3 / e2e_serial_s,
                                       "ms_per_step": 1e3 * e2e_serial_s / K3}}
         del lanes
