@@ -56,7 +56,7 @@ typedef enum {
  * pointer may be NULL); n_group must be 1 and groups <= 32 * top_k. */
 enum { MOE_SCORE_SOFTMAX = 0, MOE_SCORE_SIGMOID = 1, MOE_ROUTE_DENSE_TP = 2 };
 
-/* Limits of this build: num_experts <= 512, top_k <= 16, max_replicas <= 8,
+/* Limits of this library: num_experts <= 512, top_k <= 16, max_replicas <= 8,
  * num_ranks*slots_per_rank <= 4096 (and small enough for the routing kernel's
  * shared-memory tables, about 2000 slots at 512 experts), max_tokens <= 262144,
  * max_tokens*top_k < 2^30, hidden % 8 == 0.  With n_group > 1:
