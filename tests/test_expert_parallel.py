@@ -358,3 +358,65 @@ def test_distributed_form_with_a_group_of_one():
     p = subprocess.run([sys.executable, "-c", DIST_WORKER], env=env, stdout=subprocess.PIPE,
                        stderr=subprocess.STDOUT, text=True, timeout=600)
     assert p.returncode == 0 and "distributed ok" in p.stdout, p.stdout[-3000:]
+
+
+@pytest.mark.gpu
+def test_captured_group_step_survives_remaps():
+    # the exchange entry points allocate nothing: a whole group step captured once in a CUDA graph
+    # stays correct when the failure set changes between replays (no recapture)
+    import torch
+    from gpu_util import assert_y_close, bf16_bits, to_dev
+    from paper_2602_21140_b200 import binding as B
+
+    wl = small("dsv3", H=256)
+    world, T_list = 4, [96, 160, 33, 128]
+    inps = batches(wl, world, T_list)
+    bias = inps[0]["bias"]
+    routers = [B.MoeRouter(B.config_for_workload(wl, max_tokens=max(T_list)), inps[0]["slot_to_expert"], bias,
+                           inps[0]["slot_scale"]) for _ in range(world)]
+    rows = sum(T_list) * wl.k
+    recv = [torch.zeros((rows, wl.H), dtype=torch.bfloat16, device="cuda") for _ in range(world)]
+    counts_all = torch.zeros((world, wl.P), dtype=torch.int32, device="cuda")
+    offs = [torch.zeros(wl.P // world + 1, dtype=torch.int32, device="cuda") for _ in range(world)]
+    logits = [to_dev(i["logits"]) for i in inps]
+    x = [to_dev(i["x"], torch.bfloat16) for i in inps]
+    outs, ys = [], []
+    for g, r in enumerate(routers):
+        r.ep_attach(world, g, [b.data_ptr() for b in recv], rows)
+        o = r.alloc_outputs(T_list[g])
+        o.slot_counts = counts_all[g]                       # on one device the all-gather is a view
+        outs.append(o)
+        ys.append(torch.empty((T_list[g], wl.H), dtype=torch.bfloat16, device="cuda"))
+
+    def step():
+        for g, r in enumerate(routers):
+            r.ep_route(logits[g], outs[g])
+        for g, r in enumerate(routers):
+            r.ep_scatter(x[g], counts_all, offs[g])
+        for g, r in enumerate(routers):
+            r.ep_combine(T_list[g], ys[g])
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    for failed in [(), (7,), (7, 20), ()]:
+        for r in routers:
+            r.set_failed_ranks(failed)
+        graph.replay()
+        torch.cuda.synchronize()
+        cfg, (snd, own) = run_oracle(wl, world, inps, failed)
+        for g in range(world):
+            assert np.array_equal(outs[g].dst_row.cpu().numpy(), snd[g]["dst_row"]), (failed, g)
+            assert_y_close(bf16_bits(ys[g]), oracle.ep_combine(cfg, world, g, snd[g], own, inps[0]["slot_scale"]))
+        for d in range(world):
+            n = own[d]["recv_buf"].shape[0]
+            assert np.array_equal(bf16_bits(recv[d][:n]), own[d]["recv_buf"]), (failed, d)
+    for r in routers:
+        assert r.device_status() == 0
+        r.close()
