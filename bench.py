@@ -553,6 +553,73 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_expert_failure_sweep(args):
+    """Sec. 4.2's lost-expert sweep as a throughput experiment: for the two selection policies
+    ("every nth", "most activated") and r in 1/64 .. 1/2, fail the experts, replay the captured
+    step and report tokens/s and the load imbalance over the physical slots that still receive
+    tokens (largest slot count / mean slot count).  One JSON line, separate from the default run."""
+    import torch
+    from paper_2602_21140_b200 import binding as B
+    from paper_2602_21140_b200 import workloads as W
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    wl = W.WORKLOADS[args.workload]
+    T, K = (args.tokens or wl.T), min(args.steps, 200)
+    inp = W.make_inputs(wl, T=T)
+    bias = inp["bias"] if wl.score_func == W.SIGMOID else None
+    router = B.MoeRouter(B.config_for_workload(wl, max_tokens=T), inp["slot_to_expert"], bias,
+                         inp["slot_scale"], device=dev)
+    logits = torch.from_numpy(inp["logits"]).to(dev)
+    x = torch.from_numpy(inp["x"]).view(torch.int16).view(torch.bfloat16).to(dev)
+    out = router.alloc_outputs(T)
+    y = torch.empty((T, wl.H), dtype=torch.bfloat16, device=dev)
+    stream = torch.cuda.Stream(device=dev)
+    rows = []
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            router.dispatch(logits, x, out)
+            router.combine(out.send_buf, T, y)
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            router.dispatch(logits, x, out)
+            router.combine(out.send_buf, T, y)
+
+        def measure(label, r, mask):
+            try:
+                router.set_failed_experts(mask)
+            except B.MoeError as e:
+                rows.append({"policy": label, "r": r, "rejected": str(e)})
+                return
+            for _ in range(3):
+                graph.replay()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(K):
+                graph.replay()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            counts = out.slot_counts.cpu().numpy().astype(np.int64)
+            used = counts[counts > 0]
+            rows.append({"policy": label, "r": r, "experts_lost": int(np.asarray(mask).sum()) if mask is not None else 0,
+                         "tokens_per_s": T * K / (e0.elapsed_time(e1) * 1e-3),
+                         "us_per_step": e0.elapsed_time(e1) * 1e3 / K,
+                         "slots_used": int(used.size), "imbalance_max_over_mean": float(used.max() / used.mean())})
+
+        measure("none", 0.0, None)
+        # activation counts per logical expert with nothing failed, for the worst-case policy
+        activations = np.bincount(out.topk_ids.cpu().numpy().reshape(-1), minlength=wl.E)
+        for r in (1 / 64, 1 / 32, 1 / 16, 1 / 8, 1 / 4, 1 / 2):
+            measure("every_nth", r, W.every_nth_mask(wl.E, r))
+            measure("most_activated", r, W.most_activated_mask(activations, r))
+        router.set_failed_experts(None)
+    assert router.device_status() == 0
+    router.close()
+    print(json.dumps({"experiment": "lost experts: throughput and load imbalance against the lost fraction r",
+                      "workload": workload_name(wl, ()), "tokens": T, "steps_per_point": K, "rows": rows}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -564,7 +631,11 @@ def main():
     ap.add_argument("--tokens", type=int, default=0, help="override T (profiling captures on a smaller case)")
     ap.add_argument("--quick", action="store_true", help="a few eager steps only (for profiler captures)")
     ap.add_argument("--no-overlap", action="store_true", help="skip the two extra legs (two batches in flight, emulated multi-GPU exchange)")
+    ap.add_argument("--expert-failure-sweep", action="store_true",
+                    help="run the lost-expert sweep (throughput and load imbalance against r) instead of the benchmark")
     args = ap.parse_args()
+    if args.expert_failure_sweep:
+        return run_expert_failure_sweep(args)
     if args.impl == "reference":
         run_reference(args)
     else:
