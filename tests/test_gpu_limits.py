@@ -85,3 +85,11 @@ def test_config_limits_are_enforced():
         assert B.moe_workspace_bytes(cfg) == 0, field
     cfg = B.config_for_workload(wl, max_tokens=262144)
     assert B.moe_workspace_bytes(cfg) > 0
+
+
+@pytest.mark.parametrize("H,k", [(16384, 8), (8200, 4), (32768, 2), (12288, 16)])
+def test_rows_wider_than_one_warp_pass(H, k):
+    # rows above 16 KB are moved in several pieces per warp by the scatter and in many column
+    # chunks by the combine; widths that are not a multiple of a chunk leave a ragged last chunk
+    wl = W.Workload("widerows", T=150, H=H, E=32, k=k, R=8, S=4, score_func=W.SOFTMAX, seed=43, max_replicas=1)
+    run_and_check(wl, W.make_inputs(wl), (5,))
