@@ -442,13 +442,22 @@ def run_ours(args):
                 outs_q.append(o)
                 ys_q.append(torch.empty((Tq, wl.H), dtype=torch.bfloat16, device=dev))
 
+            vstreams = [torch.cuda.Stream(device=dev) for _ in range(Gv)]
+
+            def on_every_virtual_gpu(fn):
+                # each virtual GPU works on its own stream, as separate devices would; all of them
+                # are joined before the next phase (the ordering a collective provides between GPUs)
+                for g, r in enumerate(vr):
+                    vstreams[g].wait_stream(stream)
+                    with torch.cuda.stream(vstreams[g]):
+                        fn(g, r)
+                for g in range(Gv):
+                    stream.wait_stream(vstreams[g])
+
             def ep_step():
-                for g, r in enumerate(vr):
-                    r.ep_route(logits[g * Tq:(g + 1) * Tq], outs_q[g])
-                for g, r in enumerate(vr):
-                    r.ep_scatter(x[g * Tq:(g + 1) * Tq], counts_all, offs[g])
-                for g, r in enumerate(vr):
-                    r.ep_combine(Tq, ys_q[g])
+                on_every_virtual_gpu(lambda g, r: r.ep_route(logits[g * Tq:(g + 1) * Tq], outs_q[g]))
+                on_every_virtual_gpu(lambda g, r: r.ep_scatter(x[g * Tq:(g + 1) * Tq], counts_all, offs[g]))
+                on_every_virtual_gpu(lambda g, r: r.ep_combine(Tq, ys_q[g]))
 
             for _ in range(3):
                 ep_step()
@@ -471,8 +480,9 @@ def run_ours(args):
             same = all(torch.equal(ys_q[g], y[g * Tq:(g + 1) * Tq]) for g in range(Gv)) if wl.n_redundant == 0 else None
             ep_leg = {"value": T / (ms_ep * 1e-3), "unit": UNIT, "ms_per_step": ms_ep, "virtual_gpus": Gv,
                       "tokens_per_virtual_gpu": Tq, "y_equals_single_gpu_step": same,
-                      "what": "4 virtual GPUs on one device: route, count table, scatter into the owners' "
-                              "receive buffers, combine from them; 16 kernels per step in one graph"}
+                      "what": "4 virtual GPUs on one device, one stream each, joined between the phases: "
+                              "route, count table, scatter into the owners' receive buffers, combine from "
+                              "them; 16 kernels per step in one graph"}
             for r in vr:
                 r.close()
             del recv, outs_q, ys_q
