@@ -148,3 +148,31 @@ def test_init_without_gpu_fails_loudly():
     assert st == B.MOE_ERR_CUDA and ctx is None
     with pytest.raises(RuntimeError):
         B.MoeRouter(B.config_for_workload(wl), inp["slot_to_expert"], None, inp["slot_scale"], device="cpu")
+
+
+def test_binding_structs_match_the_header_layout(tmp_path):
+    # the ctypes mirrors of the header's structs must have the C compiler's sizes and offsets
+    import ctypes
+    import os
+    import subprocess
+    from paper_2602_21140_b200 import binding as B
+
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    fields = {"moe_config": [f for f, _ in B.moe_config._fields_],
+              "moe_dispatch_out": [f for f, _ in B.moe_dispatch_out._fields_],
+              "moe_ep_group": [f for f, _ in B.moe_ep_group._fields_]}
+    lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "moe_route.h"', 'int main(void) {']
+    for s, fs in fields.items():
+        lines.append(f'printf("{s} %zu\\n", sizeof({s}));')
+        for f in fs:
+            lines.append(f'printf("{s}.{f} %zu\\n", offsetof({s}, {f}));')
+    lines += ['return 0; }']
+    src, exe = tmp_path / "layout.c", tmp_path / "layout"
+    src.write_text("\n".join(lines))
+    subprocess.check_call(["gcc", "-I", os.path.join(root, "include"), "-o", str(exe), str(src)])
+    got = dict(line.split() for line in subprocess.check_output([str(exe)], text=True).splitlines())
+    for s in fields:
+        cls = getattr(B, s)
+        assert int(got[s]) == ctypes.sizeof(cls), s
+        for f in fields[s]:
+            assert int(got[f"{s}.{f}"]) == getattr(cls, f).offset, (s, f)
