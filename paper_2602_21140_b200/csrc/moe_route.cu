@@ -275,7 +275,9 @@ cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_
 template <int EPL, int LPT>
 cudaError_t launch_route_t(const RouteParams &p, int tiles, size_t smem, cudaStream_t st, bool pdl)
 {
-    if (smem > 48 * 1024) {
+    // the kernel also has a few hundred bytes of static shared memory: opt in to the large
+    // carve-out a little below the 48 KB default limit, not exactly at it
+    if (smem + 2048 > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(k_route<EPL, LPT>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;

@@ -93,3 +93,18 @@ def test_rows_wider_than_one_warp_pass(H, k):
     # chunks by the combine; widths that are not a multiple of a chunk leave a ragged last chunk
     wl = W.Workload("widerows", T=150, H=H, E=32, k=k, R=8, S=4, score_func=W.SOFTMAX, seed=43, max_replicas=1)
     run_and_check(wl, W.make_inputs(wl), (5,))
+
+
+@pytest.mark.parametrize("R", [83, 84, 85, 86, 87, 88])
+def test_routing_tables_around_the_default_shared_memory_limit(R):
+    # slot counts that put the routing kernel's shared-memory tables just below, at and just
+    # above the 48 KB a kernel gets without opting in to more
+    E, S, copies = 192, 7, 3
+    wl = W.Workload("smem-edge", T=244, H=584, E=E, k=3, R=R, S=S, score_func=W.SOFTMAX, seed=47,
+                    max_replicas=copies)
+    inp = W.make_inputs(dataclasses.replace(wl, max_replicas=1, R=24, S=8))   # logits / x only
+    s2e = np.full(R * S, -1, np.int32)
+    s2e[: E * copies] = np.repeat(np.arange(E), copies)      # three copies of every expert, the rest empty
+    inp["slot_to_expert"] = s2e
+    inp["slot_scale"] = np.random.default_rng(4).uniform(0.5, 1.5, R * S).astype(np.float32)
+    run_and_check(wl, inp, (1, 40))

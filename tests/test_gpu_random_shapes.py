@@ -36,8 +36,9 @@ def _draw(rng):
                 scale=float(rng.choice([1.0, 2.5])))
 
 
-def test_random_configurations_match_the_oracle():
-    rng = np.random.default_rng(20261128)
+@pytest.mark.parametrize("seed", [20261128, 3, 11])
+def test_random_configurations_match_the_oracle(seed):
+    rng = np.random.default_rng(seed)
     accepted = 0
     for trial in range(400):
         c = _draw(rng)
