@@ -184,3 +184,52 @@ def test_long_run_of_replays_with_remaps_stays_exact(name, T, replays):
     check_dispatch(out, ref)
     assert_y_close(bf16_bits(y), ref["y"])
     router.close()
+
+
+@pytest.mark.parametrize("name", ["dsv3", "qwen3"])
+def test_random_sequence_of_remaps_under_one_graph(name):
+    # every kind of remap (failed ranks, lost experts, rank order, replica map), drawn at random and
+    # applied between replays of one captured graph; a rejected remap must leave the state as it was
+    import dataclasses
+    wl = dataclasses.replace(W.WORKLOADS[name], H=64)
+    T = 300
+    inp = W.make_inputs(wl, T=T)
+    bias = inp["bias"] if wl.score_func == W.SIGMOID else None
+    router = make_router(wl, inp, max_tokens=T)
+    logits, x = to_dev(inp["logits"]), to_dev(inp["x"], torch.bfloat16)
+    graph, out, y = _capture(router, logits, x, T)
+    rng = np.random.default_rng(5)
+    failed, lost, order, s2e = (), np.zeros(wl.E, np.uint8), None, inp["slot_to_expert"].copy()
+    applied = rejected = 0
+    for _ in range(120):
+        op = int(rng.integers(0, 4))
+        nf, nl, no, ns = failed, lost, order, s2e
+        try:
+            if op == 0:
+                nf = tuple(int(r) for r in rng.choice(wl.R, int(rng.integers(0, max(2, wl.R // 3))), replace=False))
+                router.set_failed_ranks(nf)
+            elif op == 1:
+                nl = (rng.random(wl.E) < rng.choice([0.0, 0.05, 0.3])).astype(np.uint8)
+                router.set_failed_experts(nl)
+            elif op == 2:
+                alive = [r for r in range(wl.R) if r not in failed]
+                no = [int(r) for r in rng.permutation(alive)] if rng.random() < 0.7 else None
+                router.set_rank_order(no if no is not None else [])
+            else:
+                ns = s2e.copy()
+                i, j = rng.integers(0, wl.P, 2)
+                ns[i], ns[j] = ns[j], ns[i]
+                router.update_replica_map(ns)
+            failed, lost, order, s2e = nf, nl, no, ns
+            applied += 1
+        except B.MoeError:
+            rejected += 1
+        graph.replay()
+        torch.cuda.synchronize()
+        assert router.device_status() == 0
+        ref = oracle.dispatch(oracle_cfg(wl), s2e, failed, bias, inp["logits"], inp["x"], lost, order)
+        check_dispatch(out, ref)
+        assert_y_close(bf16_bits(y), oracle.combine(ref["send_buf"], ref["dst_row"], ref["topk_weights"],
+                                                    ref["topk_slot"], inp["slot_scale"]))
+    assert applied > 60 and rejected > 0
+    router.close()
