@@ -251,7 +251,11 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned full = 0xffffffffu;
 
-    pdl_enter();
+    // Wait for the previous kernel first and only then let the scatter be scheduled: the scatter
+    // requests its first x rows before its own wait, which is safe only once whatever produced x
+    // (a kernel before this one) is known to have completed.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (tid == 0) {
         // ticket (low word) and epoch (high word) share one 64-bit word: a single atomic add
         // takes the ticket and reads the epoch (the ticket never carries: it is reset every step)

@@ -51,13 +51,14 @@ __global__ void __launch_bounds__(kScatterThreads) k_scatter_vec(ScatterParams p
 {
     constexpr int kChunk = 32 * UNROLL;
     const unsigned full = 0xffffffffu;
-    pdl_enter();
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int lane = lane_id();
     const int chunks = (p.hv + kChunk - 1) / kChunk;
     const long long items = (long long)p.T * chunks;
     const long long warp0 = (long long)blockIdx.x * (kScatterThreads / 32) + (threadIdx.x >> 5);
     const long long nwarps = (long long)gridDim.x * (kScatterThreads / 32);
 
+    bool waited = false;
     for (long long it = warp0; it < items; it += nwarps) {
         const int t = (int)(it / chunks);
         const int c0 = (int)(it % chunks) * kChunk + lane;
@@ -66,6 +67,13 @@ __global__ void __launch_bounds__(kScatterThreads) k_scatter_vec(ScatterParams p
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u)
             if (c0 + 32 * u < p.hv) v[u] = ld_stream_v4(src + c0 + 32 * u);
+        if (!waited) {
+            // x is an input of the dispatch, not a product of the routing kernel: the first rows
+            // are requested while that kernel is still finishing, and only the destinations
+            // (which it computes) wait for it
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            waited = true;
+        }
         const int row = resolve_row(p, t, lane, it % chunks == 0);
         for (int j = 0; j < p.k; ++j) {
             const int r = __shfl_sync(full, row, j);
