@@ -38,7 +38,7 @@ E2E_STEPS_IN_FLIGHT = int(os.environ.get("MOE_BENCH_E2E_IN_FLIGHT", "2"))   # ho
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from ncu captures of
 # the kernels as they stand at the DSv3 shape (summaries under profiles/); None when a kernel
 # changed after its last capture.
-NCU_TRAFFIC_BYTES = {"k_scatter": 998_273_792, "k_combine": 1_050_535_424}
+NCU_TRAFFIC_BYTES = {"k_scatter": 998_612_992, "k_combine": 1_051_182_336}
 
 
 def env_rank():
