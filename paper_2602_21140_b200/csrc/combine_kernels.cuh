@@ -165,7 +165,7 @@ __global__ void __launch_bounds__(kCombineBulkMaxWarps * 32) k_combine_bulk(Comb
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncwarp();
-    pdl_enter();                                           // the ring is set up; now wait for the inputs
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     const int chunks = (p.hv + kChunkV - 1) / kChunkV;
     const long long items = (long long)p.T * chunks;
@@ -174,11 +174,14 @@ __global__ void __launch_bounds__(kCombineBulkMaxWarps * 32) k_combine_bulk(Comb
     const long long per = items / nwarps, extra = items % nwarps;      // contiguous, balanced runs
     const long long first = wid * per + (wid < extra ? wid : extra);
     const int n_mine = (int)(per + (wid < extra ? 1 : 0));
-    if (n_mine == 0) return;
 
     // issuing side: token / chunk / stage of the next item to request (lane j < k owns row j)
     int it_tok = (int)(first / chunks), it_chunk = (int)(first % chunks), it_stage = 0;
     const uint4 *row, *row_next; float coef, coef_next;
+    // The ring is set up and the run is known; only now wait for the previous kernel (the one
+    // that filled the rows and wrote dst_row).
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (n_mine == 0) return;
     combine_fetch_index(p, it_tok, lane, row, coef);
     combine_fetch_index(p, it_tok + 1, lane, row_next, coef_next);
 
