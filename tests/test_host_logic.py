@@ -176,3 +176,20 @@ def test_binding_structs_match_the_header_layout(tmp_path):
         assert int(got[s]) == ctypes.sizeof(cls), s
         for f in fields[s]:
             assert int(got[f"{s}.{f}"]) == getattr(cls, f).offset, (s, f)
+
+
+def test_benchmark_byte_accounting():
+    # the roofline numerator: rows moved by the method (read x once, write k copies; read k rows,
+    # write one) plus the small index traffic, per token and per step at the DeepSeek-V3 shape
+    import bench
+    from paper_2602_21140_b200 import workloads as W
+    wl = W.WORKLOADS["dsv3"]
+    per_kernel = bench.algorithmic_bytes(wl, wl.T)
+    rows = (2 * wl.k + 2) * 2 * wl.H                       # 18 rows of 14 336 bytes
+    assert rows == 258048
+    per_token = sum(per_kernel.values()) // wl.T
+    assert per_token == rows + 4 * wl.E + 52 * wl.k        # 1 024 B of logits, 416 B of indices
+    assert per_token == 259488
+    assert per_kernel["k_scatter"] > per_kernel["k_combine"] > 100 * per_kernel["k_route"]
+    tiny = W.WORKLOADS["tiny"]
+    assert bench.algorithmic_bytes(tiny, 0) == {"k_route": 0, "k_scatter": 0, "k_combine": 0}
