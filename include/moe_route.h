@@ -271,8 +271,9 @@ moe_status moe_ep_route(moe_ctx *ctx, const float *logits, int32_t T, const moe_
  *   recv_slot_offsets device [P/world + 1] i32 out: first row of each of this GPU's slots in
  *                     its own receive buffer, last entry = rows received
  * Writes out->dst_row of the preceding moe_ep_route.  If the rows sent to a GPU exceed
- * recv_rows the surplus rows are not written and that GPU's device status becomes
- * MOE_ERR_CAPACITY (moe_get_device_status).  Allocates nothing, does not synchronise.
+ * recv_rows the surplus rows are not written, their dst_row is -1 (moe_ep_combine then
+ * lets them contribute zero and reads nothing out of range) and that GPU's device status
+ * becomes MOE_ERR_CAPACITY (moe_get_device_status).  Allocates nothing, does not synchronise.
  */
 moe_status moe_ep_scatter(moe_ctx *ctx, const void *x, int32_t T, const int32_t *counts_all,
                           int32_t *recv_slot_offsets, void *cuda_stream);
@@ -320,6 +321,46 @@ moe_status moe_step_host_async(moe_ctx *ctx, const float *logits_host, const voi
                                void *y_dev, void *y_host, void *cuda_stream);
 
 /*
+ * moe_set_tuning — override one launch choice of a context (no counterpart in the paper).
+ * A context picks kernel variants and launch shapes from its shape alone; nothing in the
+ * process environment influences it.  This call replaces one choice, for measurements and
+ * for tests of the non-default kernels.  `value` = -1 restores the automatic choice; a value
+ * a kernel cannot honour is clamped to the nearest one it can.  The call waits for the
+ * device, may reallocate the scan scratch (the two routing options) and must not be made
+ * while a stream is capturing or between a dispatch and its combine.  Graphs captured
+ * before the call keep the launch shapes they were captured with.
+ */
+typedef enum {
+    MOE_TUNE_PDL = 0,                     /* 1 (default): programmatic dependent launch; 0: plain launches      */
+    MOE_TUNE_SCATTER_IMPL = 1,            /* 0 (default): 128-bit vector copies; 1: bulk-copy ring               */
+    MOE_TUNE_SCATTER_BULK_STAGES = 2,     /* bulk-copy scatter: ring depth, 1..8 (default 4)                     */
+    MOE_TUNE_SCATTER_BULK_CTAS_PER_SM = 3,/* bulk-copy scatter: one-warp CTAs per SM (default: as many as fit)   */
+    MOE_TUNE_SCATTER_BLOCKS_PER_SM = 4,   /* vector scatter: grid cap in CTAs per SM (default 8)                 */
+    MOE_TUNE_SCATTER_UNROLL = 5,          /* vector scatter: 16-byte units per lane, one of 4, 8, 16, 28, 32     */
+    MOE_TUNE_COMBINE_IMPL = 6,            /* 1 (default): bulk-copy ring; 0: vector loads                        */
+    MOE_TUNE_COMBINE_CHUNK = 7,           /* ring combine: 16-byte units per lane and row chunk, 1, 2 or 4       */
+    MOE_TUNE_COMBINE_STAGES = 8,          /* ring combine: stages per warp, 2..8                                 */
+    MOE_TUNE_COMBINE_WARPS = 9,           /* ring combine: warps per CTA, 1..8                                   */
+    MOE_TUNE_COMBINE_CTAS_PER_SM = 10,    /* ring combine: CTAs per SM (default: as many as fit)                 */
+    MOE_TUNE_ROUTE_LANES_PER_TOKEN = 11,  /* routing: 8 or 16 lanes of a warp per token                          */
+    MOE_TUNE_ROUTE_TOKENS_PER_TILE = 12,  /* routing: tokens per tile (default: max_tokens / 148, at least 32)   */
+    MOE_TUNE_SPIN_LIMIT = 13              /* polls before a bounded device wait gives up (default 1 << 20)       */
+} moe_tuning_option;
+
+moe_status moe_set_tuning(moe_ctx *ctx, int32_t option, int32_t value);
+
+/*
+ * moe_debug_skip_ticket — test hook for the give-up path of the bounded device waits (no
+ * counterpart in the paper).  Advances the tile ticket of the NEXT routing kernel by one, so
+ * that no CTA ever routes the step's first tile: every other tile then waits for a
+ * publication that never comes, runs out of polls (MOE_TUNE_SPIN_LIMIT), sets the status
+ * word to MOE_ERR_DEVICE_TIMEOUT and returns.  Nothing faults and nothing waits without a
+ * limit.  The outputs of that step are incomplete: follow it only by moe_get_device_status,
+ * which re-arms the context.  Waits for the device.
+ */
+moe_status moe_debug_skip_ticket(moe_ctx *ctx);
+
+/*
  * moe_set_timing_event — measurement hook (no counterpart in the paper).
  * `cuda_event` is a cudaEvent_t created by the caller with timing enabled, or
  * NULL to switch the hook off.  While set, every moe_dispatch records it on
@@ -333,7 +374,10 @@ moe_status moe_set_timing_event(moe_ctx *ctx, void *cuda_event);
  * moe_get_device_status — synchronises the device and reports whether any
  * kernel of this context gave up on a bounded wait or met a token with fewer
  * than k selectable experts (possible only with -inf logits).  Writes the
- * status to *code, clears it and resets the scan scratch.  Never on the hot path.
+ * status to *code, clears it and re-arms the scan scratch.  Never on the hot path.
+ * After a wait gave up (MOE_ERR_DEVICE_TIMEOUT) the step's outputs are incomplete:
+ * assignments that were not placed have dst_row = -1 and contribute zero to a combine;
+ * until this call has re-armed the context, later routing kernels route nothing.
  */
 moe_status moe_get_device_status(moe_ctx *ctx, int32_t *code);
 
@@ -376,8 +420,12 @@ moe_status moe_plan_routing_state(const moe_config *cfg, const int32_t *slot_to_
  * Limits: P <= 512 and n_assign <= 262144; anything larger returns
  * MOE_ERR_CAPACITY and launches nothing.  n_assign = 0 writes zero counts.
  * The first call on each device looks up the scratch array's device address
- * (one runtime query, no allocation); make that first call before starting any
- * stream capture.  All calls on a device share the one array: the function
+ * (one runtime query); make that first call before starting any stream capture.
+ * With lazy module loading that first call is also the moment the driver loads
+ * this function's device code, scratch array included, onto the device, which
+ * takes device memory: make it at start-up, BEFORE the process claims the rest of
+ * HBM (a warm-up call with n_assign = 0 is enough).  Every later call allocates
+ * nothing.  All calls on a device share the one array: the function
  * rewrites every word it reads, so leftovers of earlier calls are harmless,
  * but two calls that overlap on the GPU (different streams without ordering)
  * race on it.  Work is enqueued on `cuda_stream`; the call does not wait.

@@ -34,6 +34,11 @@ MOE_ERR_DEVICE_TIMEOUT = 5
 MOE_SCORE_SOFTMAX = 0
 MOE_SCORE_SIGMOID = 1
 MOE_ROUTE_DENSE_TP = 2
+# options of moe_set_tuning (include/moe_route.h, moe_tuning_option)
+(MOE_TUNE_PDL, MOE_TUNE_SCATTER_IMPL, MOE_TUNE_SCATTER_BULK_STAGES, MOE_TUNE_SCATTER_BULK_CTAS_PER_SM,
+ MOE_TUNE_SCATTER_BLOCKS_PER_SM, MOE_TUNE_SCATTER_UNROLL, MOE_TUNE_COMBINE_IMPL, MOE_TUNE_COMBINE_CHUNK,
+ MOE_TUNE_COMBINE_STAGES, MOE_TUNE_COMBINE_WARPS, MOE_TUNE_COMBINE_CTAS_PER_SM,
+ MOE_TUNE_ROUTE_LANES_PER_TOKEN, MOE_TUNE_ROUTE_TOKENS_PER_TILE, MOE_TUNE_SPIN_LIMIT) = range(14)
 
 EXPORTED_SYMBOLS = (
     "moe_route_init", "moe_set_failed_ranks", "moe_update_replica_map", "moe_dispatch",
@@ -41,6 +46,7 @@ EXPORTED_SYMBOLS = (
     "moe_workspace_bytes", "moe_route_destroy", "moe_status_string", "moe_permute_static",
     "moe_set_failed_experts", "moe_compact_ranks", "moe_set_rank_order",
     "moe_ep_attach", "moe_ep_route", "moe_ep_scatter", "moe_ep_combine", "moe_ep_plan_host",
+    "moe_set_tuning", "moe_debug_skip_ticket",
 )
 
 
@@ -128,6 +134,10 @@ def _lib():
         lib.moe_ep_combine.argtypes = [vp, i32, vp, vp]
         lib.moe_ep_plan_host.restype = ctypes.c_int
         lib.moe_ep_plan_host.argtypes = [vp, i32, i32, i32, vp, vp]
+        lib.moe_set_tuning.restype = ctypes.c_int
+        lib.moe_set_tuning.argtypes = [vp, i32, i32]
+        lib.moe_debug_skip_ticket.restype = ctypes.c_int
+        lib.moe_debug_skip_ticket.argtypes = [vp]
         lib.moe_status_string.restype = ctypes.c_char_p
         lib.moe_status_string.argtypes = [ctypes.c_int]
         _lib_handle = lib
@@ -250,6 +260,14 @@ def moe_step_host_async(ctx, logits_host_ptr: int, x_host_ptr: int, T: int, out:
 
 def moe_set_timing_event(ctx, cuda_event: int) -> int:
     return _lib().moe_set_timing_event(ctx, ctypes.c_void_p(cuda_event) if cuda_event else None)
+
+
+def moe_set_tuning(ctx, option: int, value: int) -> int:
+    return _lib().moe_set_tuning(ctx, int(option), int(value))
+
+
+def moe_debug_skip_ticket(ctx) -> int:
+    return _lib().moe_debug_skip_ticket(ctx)
 
 
 def moe_get_device_status(ctx):
@@ -482,6 +500,12 @@ class MoeRouter:
         st = moe_set_timing_event(self._ctx, handle)
         if st != MOE_OK:
             raise MoeError(st, "moe_set_timing_event")
+
+    def set_tuning(self, option: int, value: int) -> None:
+        """Override one launch choice of the context (see moe_tuning_option); -1 = automatic."""
+        st = moe_set_tuning(self._ctx, option, value)
+        if st != MOE_OK:
+            raise MoeError(st, "moe_set_tuning")
 
     def device_status(self) -> int:
         st, code = moe_get_device_status(self._ctx)

@@ -24,6 +24,10 @@ struct CombineParams {
     // that buffer.  NULL = every row is in `buf`.
     const uint4 *const *peer_bufs;
     int slots_per_gpu;
+    int P;                       // physical slots
+    long long row_limit;         // rows a source buffer holds: T*k, or the receive-buffer capacity
+    const uint4 *zero_row;       // [H/8] zeros: stands in for a row that was not placed
+    unsigned spin_limit;         // polls before a bounded wait gives up
 };
 
 constexpr int kCombineThreads = 256;
@@ -69,8 +73,14 @@ __global__ void __launch_bounds__(kCombineThreads) k_combine_vec(CombineParams p
         int my_row = 0; float my_coef = 0.0f;
         if (lane < k) {
             const size_t i = (size_t)t * k + lane;
-            my_row = __ldg(p.dst_row + i);
-            my_coef = __fmul_rn(__ldg(p.topk_weights + i), __ldg(p.slot_scale + __ldg(p.topk_slot + i)));
+            const int slot = __ldg(p.topk_slot + i);
+            const int r = __ldg(p.dst_row + i);
+            if ((unsigned)slot < (unsigned)p.P && r >= 0 && r < p.row_limit) {
+                my_row = r;
+                my_coef = __fmul_rn(__ldg(p.topk_weights + i), __ldg(p.slot_scale + slot));
+            } else {
+                my_row = -1;                               // not placed: contributes nothing
+            }
         }
         float acc[kCombineUnroll][8];
 #pragma unroll
@@ -83,7 +93,7 @@ __global__ void __launch_bounds__(kCombineThreads) k_combine_vec(CombineParams p
 #pragma unroll
             for (int j = 0; j < K; ++j) {
                 const int r = __shfl_sync(full, my_row, j);
-                const uint4 *src = p.buf + (size_t)r * p.hv;
+                const uint4 *src = (r >= 0) ? p.buf + (size_t)r * p.hv : p.zero_row;
 #pragma unroll
                 for (int u = 0; u < kCombineUnroll; ++u)
                     if (c0 + 32 * u < p.hv) v[j][u] = ld_stream_v4(src + c0 + 32 * u);
@@ -99,7 +109,7 @@ __global__ void __launch_bounds__(kCombineThreads) k_combine_vec(CombineParams p
             for (int j = 0; j < k; ++j) {
                 const int r = __shfl_sync(full, my_row, j);
                 const float c = __shfl_sync(full, my_coef, j);
-                const uint4 *src = p.buf + (size_t)r * p.hv;
+                const uint4 *src = (r >= 0) ? p.buf + (size_t)r * p.hv : p.zero_row;
 #pragma unroll
                 for (int u = 0; u < kCombineUnroll; ++u)
                     if (c0 + 32 * u < p.hv) fma_bf16x8(acc[u], ld_stream_v4(src + c0 + 32 * u), c);
@@ -126,13 +136,18 @@ constexpr int kCombineBulkMaxWarps = 8;   // warps per CTA (blockDim.x / 32), ea
 __device__ __forceinline__ void combine_fetch_index(const CombineParams &p, int t, int lane,
                                                     const uint4 *&row, float &coef)
 {
-    row = p.buf; coef = 0.0f;
+    // An assignment whose slot or row is out of range (a row that did not fit its receive buffer,
+    // or indices left behind by a routing kernel that gave up) reads the row of zeros instead.
+    row = p.zero_row; coef = 0.0f;
     if (lane < p.k && t < p.T) {
         const size_t i = (size_t)t * p.k + lane;
         const int slot = __ldg(p.topk_slot + i);
-        const uint4 *base = p.peer_bufs ? p.peer_bufs[slot / p.slots_per_gpu] : p.buf;
-        row = base + (size_t)__ldg(p.dst_row + i) * p.hv;
-        coef = __fmul_rn(__ldg(p.topk_weights + i), __ldg(p.slot_scale + slot));
+        const int r = __ldg(p.dst_row + i);
+        if ((unsigned)slot < (unsigned)p.P && r >= 0 && r < p.row_limit) {
+            const uint4 *base = p.peer_bufs ? p.peer_bufs[slot / p.slots_per_gpu] : p.buf;
+            row = base + (size_t)r * p.hv;
+            coef = __fmul_rn(__ldg(p.topk_weights + i), __ldg(p.slot_scale + slot));
+        }
     }
 }
 
@@ -215,7 +230,7 @@ __global__ void __launch_bounds__(kCombineBulkMaxWarps * 32) k_combine_bulk(Comb
         if (n + stages - 1 < n_mine) issue();              // refills the stage consumed at n-1
         unsigned spins = 0;
         while (!mbar_try_wait(&full[stage], parity)) {
-            if (++spins > kSpinLimit) { ok = false; break; }
+            if (++spins > p.spin_limit) { ok = false; break; }
         }
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
@@ -261,11 +276,11 @@ __global__ void __launch_bounds__(kCombineBulkMaxWarps * 32) k_combine_bulk(Comb
     }
     if (!ok) {
         if (lane == 0) report_status(ctl, kDevTimeout);
-        // copies issued for items n .. n+stages-2 may still be landing in this CTA's shared
+        // copies issued for items n .. n+stages-1 may still be landing in this CTA's shared
         // memory: give each a bounded chance to finish before the memory is released
-        for (int m = n; m < min(n_mine, n + stages - 1); ++m) {
+        for (int m = n; m < min(n_mine, n + stages); ++m) {
             unsigned spins = 0;
-            while (!mbar_try_wait(&full[m % stages], (unsigned)(m / stages) & 1u) && ++spins < kSpinLimit) {}
+            while (!mbar_try_wait(&full[m % stages], (unsigned)(m / stages) & 1u) && ++spins < p.spin_limit) {}
         }
     }
 }

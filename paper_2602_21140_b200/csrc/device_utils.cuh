@@ -12,9 +12,10 @@ constexpr int kDevInsufficientExperts = 3;   // a token met fewer than k selecta
 constexpr int kDevCapacity = 4;              // rows of an exchange did not fit the receive buffer
 constexpr int kDevTimeout = 5;               // a bounded wait gave up
 
-// Bounded waits: polls before a waiter gives up, and the back-off between polls.
+// Bounded waits: default number of polls before a waiter gives up (a context may carry
+// another limit), and the back-off between polls of a flag in global memory.
 // 1<<20 polls of >= 64 ns is well over 50 ms, far longer than any healthy step.
-constexpr unsigned kSpinLimit = 1u << 20;
+constexpr unsigned kDefaultSpinLimit = 1u << 20;
 constexpr unsigned kSpinSleepNs = 64;
 
 struct Control {
@@ -59,6 +60,18 @@ __device__ __forceinline__ unsigned ld_relaxed_u32(const unsigned *p)
     unsigned v;
     asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
+}
+
+__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p)
+{
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+__device__ __forceinline__ void st_relaxed_u32(unsigned *p, unsigned v)
+{
+    asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
 __device__ __forceinline__ int ld_relaxed_s32(const int *p)

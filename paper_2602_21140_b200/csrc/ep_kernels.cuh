@@ -58,7 +58,7 @@ __global__ void __launch_bounds__(kEpPlanThreads) k_ep_plan(EpPlanParams p)
 struct EpScatterParams {
     const uint4 *x;               // [T, H/8]
     uint4 *const *peer_bufs;      // device [G]: every GPU's receive buffer as seen from this GPU
-    int T, k, hv, spg;
+    int T, k, hv, spg, P;
     long long recv_rows;
     const int32_t *topk_slot;     // [T,k]
     const int32_t *src_base;      // [P]
@@ -70,7 +70,8 @@ constexpr int kEpScatterThreads = 256;
 
 // A warp takes (token, piece of 32*UNROLL 16-byte units of the row), loads the piece once
 // and stores it into the k owners' buffers.  A row that would fall outside the owner's
-// buffer is not written (the owner's plan kernel reports the overflow).
+// buffer is not written and its dst_row becomes -1 (the owner's plan kernel reports the
+// overflow; the combine treats the assignment as contributing zero).
 template <int UNROLL>
 __global__ void __launch_bounds__(kEpScatterThreads) k_ep_scatter(EpScatterParams p)
 {
@@ -95,9 +96,14 @@ __global__ void __launch_bounds__(kEpScatterThreads) k_ep_scatter(EpScatterParam
         if (lane < p.k) {
             const size_t i = (size_t)t * p.k + lane;
             const int slot = __ldg(p.topk_slot + i);
-            const int row = __ldg(p.src_base + slot) + __ldg(p.pos_in_slot + i);
-            if (it % chunks == 0) p.dst_row[i] = row;
-            if (row < p.recv_rows)
+            // 64-bit: the clamped base of a hopelessly overflowed buffer plus a rank must not wrap
+            long long row = -1;
+            if ((unsigned)slot < (unsigned)p.P)
+                row = (long long)__ldg(p.src_base + slot) + __ldg(p.pos_in_slot + i);
+            const bool fits = row >= 0 && row < p.recv_rows;
+            // a row that does not fit is recorded as not placed (-1): the combine skips it
+            if (it % chunks == 0) p.dst_row[i] = fits ? (int)row : -1;
+            if (fits)
                 dst_bits = reinterpret_cast<unsigned long long>(p.peer_bufs[slot / p.spg] + (size_t)row * p.hv);
         }
         for (int j = 0; j < p.k; ++j) {

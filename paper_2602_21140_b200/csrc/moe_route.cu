@@ -7,8 +7,8 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
-#include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -27,6 +27,8 @@ constexpr int kMaxReplicas = 8;
 constexpr int kMaxSlots = 4096;
 constexpr int kStagingSlots = 16;
 constexpr size_t kMaxSmem = 227 * 1024;
+constexpr int kRouteTileTarget = 148;   // tiles of a full step: one per SM of a B200
+constexpr int kNumTuning = MOE_TUNE_SPIN_LIMIT + 1;
 
 // Shape-derived launch constants.
 struct Derived {
@@ -39,23 +41,19 @@ struct Derived {
     int expert_words;      // words of the failed-expert bitmap
     int state_words;       // words of the whole routing-state blob
     int tokens_per_block;  // routing tile
+    int p_pad;             // P rounded up to a multiple of 8 (row pitch of the per-tile counts)
 };
-
-int env_int(const char *name, int dflt)
-{
-    const char *v = std::getenv(name);
-    return (v && *v) ? std::atoi(v) : dflt;
-}
 
 bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
 
-bool derive(const moe_config *c, Derived *d)
+// `want_lpt` (8 or 16) and `want_tile` (tokens) override the automatic choices; 0 = automatic.
+bool derive(const moe_config *c, Derived *d, int want_lpt = 0, int want_tile = 0)
 {
     if (!c) return false;
     if (c->num_experts < 1 || c->num_experts > kMaxExperts) return false;
     if (c->top_k < 1 || c->top_k > kMaxTopK || c->top_k > c->num_experts) return false;
     if (c->hidden < 8 || c->hidden % 8 != 0) return false;
-    if (c->max_tokens < 1) return false;
+    if (c->max_tokens < 1 || c->max_tokens > 262144) return false;
     if (c->num_ranks < 1 || c->slots_per_rank < 1) return false;
     const long long P = (long long)c->num_ranks * c->slots_per_rank;
     if (P > kMaxSlots) return false;
@@ -87,7 +85,6 @@ bool derive(const moe_config *c, Derived *d)
     }
     // 16 lanes per token above 64 experts: twice the warps in flight for the same work,
     // which measured faster than 8 lanes (the kernel is issue/latency bound)
-    int want_lpt = env_int("MOE_ROUTE_LPT", 0);
     if (want_lpt != 8 && want_lpt != 16) want_lpt = (d->E > 64) ? 16 : 0;
     for (int lpt : kLpt) {
         if (d->epl || d->k > lpt || (want_lpt && lpt < want_lpt)) continue;
@@ -108,13 +105,20 @@ bool derive(const moe_config *c, Derived *d)
     d->rank_words = (d->R + 31) / 32;
     d->expert_words = (d->E + 31) / 32;
     d->state_words = kStateHeaderWords + d->rank_words + d->expert_words + d->E * d->max_rep + d->P;
-    // routing tile: a power of two, grown with max_tokens so that a step has <= 128 tiles
-    d->tokens_per_block = 32;
-    while ((c->max_tokens + d->tokens_per_block - 1) / d->tokens_per_block > kMaxRouteTiles)
-        d->tokens_per_block *= 2;
-    if (d->tokens_per_block > 2048) return false;      // max_tokens <= 262144
-    if (route_smem_bytes(d->E, d->max_rep, d->tokens_per_block, d->k, d->P) > kMaxSmem - 1024)
+    d->p_pad = (d->P + 7) & ~7;
+    // Routing tile: a full step should have one tile per SM (a tile is one CTA, and all tiles of
+    // a step run in one wave), but never fewer than 32 tokens; a multiple of the tokens a warp
+    // routes at once.  Halved until the tile's tables fit in shared memory.
+    const int per_warp = 32 / d->lpt;
+    int tile = want_tile > 0 ? want_tile : std::max(32, (c->max_tokens + kRouteTileTarget - 1) / kRouteTileTarget);
+    tile = (tile + per_warp - 1) / per_warp * per_warp;
+    while (tile > per_warp &&
+           (route_smem_bytes(d->E, d->max_rep, tile, d->k, d->P) > kMaxSmem - 1024 || (long long)tile * d->k > 65535))
+        tile = (tile / 2 + per_warp - 1) / per_warp * per_warp;
+    if (route_smem_bytes(d->E, d->max_rep, tile, d->k, d->P) > kMaxSmem - 1024 || (long long)tile * d->k > 65535)
         return false;
+    d->tokens_per_block = tile;
+    if ((c->max_tokens + tile - 1) / tile > kMaxRouteTiles) return false;
     return true;
 }
 
@@ -209,18 +213,24 @@ struct moe_ctx {
     int n_listed;                      // leading entries given by the caller; the rest own no rows
     // device state
     int32_t *d_state;
+    int32_t *d_live;           // live-replica lists derived from d_state (k_derive_live)
     float *d_bias;
     float *d_slot_scale;
-    unsigned long long *d_desc;
+    uint16_t *d_tile_counts;   // [tiles][p_pad] per-tile, per-slot counts of the running step
+    unsigned *d_tile_flag;     // [tiles] epoch of the step that published the row
+    size_t scan_tiles;         // rows the two arrays above were allocated for
     moe::Control *d_ctl;
     int32_t *d_pos;
+    uint4 *d_zero_row;         // [H/8] zeros: source of an assignment that was not placed
     size_t device_bytes;
     // pinned staging ring for stream-ordered remaps
     int32_t *h_stage[kStagingSlots];
     cudaEvent_t stage_done[kStagingSlots];
     bool stage_used[kStagingSlots];
     unsigned stage_next;
-    // launch choices
+    // launch choices (configure_launch); tune[] holds the overrides of moe_set_tuning, -1 = automatic
+    int tune[kNumTuning];
+    unsigned spin_limit;   // polls before a bounded device wait gives up
     bool pdl;              // launch with the programmatic-dependent-launch attribute
     int scatter_impl;      // 0 = vector, 1 = bulk copies
     int bulk_stages, bulk_ctas_per_sm;
@@ -250,10 +260,12 @@ size_t device_bytes_for(const Derived &d, int max_tokens)
     const size_t tiles = ((size_t)max_tokens + d.tokens_per_block - 1) / d.tokens_per_block;
     size_t b = 0;
     b += (size_t)d.state_words * 4;
+    b += (size_t)d.E * (1 + d.max_rep) * 4;
     b += (size_t)d.E * 4 + (size_t)d.P * 4;
-    b += tiles * d.P * sizeof(unsigned long long);
+    b += tiles * d.p_pad * sizeof(uint16_t) + tiles * sizeof(unsigned);
     b += sizeof(moe::Control);
     b += (size_t)max_tokens * d.k * 4;
+    b += (size_t)d.H * 2;
     return b;
 }
 
@@ -327,7 +339,8 @@ cudaError_t launch_combine(const CombineParams &p, int blocks, cudaStream_t st)
     return cudaGetLastError();
 }
 
-// The routing kernel of a dispatch (a1..a9 except the final row addition).
+// The routing kernel of a dispatch: everything from the gate to the per-slot offsets and the
+// rank of every assignment inside its slot (the scatter adds the slot's offset).
 cudaError_t enqueue_route(moe_ctx *ctx, const float *logits, int32_t T, const moe_dispatch_out *out,
                           cudaStream_t st)
 {
@@ -337,14 +350,14 @@ cudaError_t enqueue_route(moe_ctx *ctx, const float *logits, int32_t T, const mo
     rp.max_rep = d.max_rep; rp.score_func = ctx->cfg.score_func; rp.n_group = ctx->cfg.n_group;
     rp.topk_group = ctx->cfg.topk_group; rp.lanes_per_group = d.lanes_per_group;
     rp.group_m = d.group_m; rp.route_scale = ctx->cfg.route_scale;
-    rp.tokens_per_block = d.tokens_per_block; rp.rank_words = d.rank_words;
-    rp.expert_words = d.expert_words;
-    rp.state = ctx->d_state; rp.bias = ctx->d_bias;
+    rp.tokens_per_block = d.tokens_per_block; rp.p_pad = d.p_pad; rp.rank_words = d.rank_words;
+    rp.expert_words = d.expert_words; rp.spin_limit = ctx->spin_limit;
+    rp.state = ctx->d_state; rp.live = ctx->d_live; rp.bias = ctx->d_bias;
     rp.topk_ids = out->topk_ids; rp.topk_weights = out->topk_weights; rp.topk_slot = out->topk_slot;
     rp.pos_in_slot = ctx->d_pos;
     rp.slot_counts = out->slot_counts; rp.slot_offsets = out->slot_offsets;
     rp.rank_counts = out->rank_counts; rp.rank_offsets = out->rank_offsets;
-    rp.desc = ctx->d_desc; rp.ctl = ctx->d_ctl;
+    rp.tile_counts = ctx->d_tile_counts; rp.tile_flag = ctx->d_tile_flag; rp.ctl = ctx->d_ctl;
     const int tiles = (T + d.tokens_per_block - 1) / d.tokens_per_block;
     return launch_route(d.epl, d.lpt, rp, tiles, ctx->route_smem, st, ctx->pdl);
 }
@@ -379,6 +392,18 @@ moe_status enqueue_combine_bulk(moe_ctx *ctx, const CombineParams &cp, cudaStrea
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Rebuild the live-replica lists from the bitmaps and the replica table, on the stream,
+// behind the state copy that precedes it.
+moe_status enqueue_derive(moe_ctx *ctx, cudaStream_t st)
+{
+    const Derived &d = ctx->d;
+    DeriveParams dp;
+    dp.state = ctx->d_state; dp.E = d.E; dp.S = d.S; dp.max_rep = d.max_rep;
+    dp.rank_words = d.rank_words; dp.expert_words = d.expert_words; dp.live = ctx->d_live;
+    k_derive_live<<<(d.E + kDeriveThreads - 1) / kDeriveThreads, kDeriveThreads, 0, st>>>(dp);
+    return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
 // Copy `words` leading words of `blob` to the device state through a pinned
 // staging slot, ordered on `st`.  A slot is reused only after its copy has run.
 moe_status push_state(moe_ctx *ctx, const std::vector<int32_t> &blob, int words, cudaStream_t st)
@@ -393,7 +418,7 @@ moe_status push_state(moe_ctx *ctx, const std::vector<int32_t> &blob, int words,
     if (cudaEventRecord(ctx->stage_done[s], st) != cudaSuccess) return MOE_ERR_CUDA;
     ctx->stage_used[s] = true;
     ctx->stage_next++;
-    return MOE_OK;
+    return enqueue_derive(ctx, st);
 }
 
 bool stream_is_capturing(cudaStream_t st)
@@ -403,11 +428,108 @@ bool stream_is_capturing(cudaStream_t st)
     return cs != cudaStreamCaptureStatusNone;
 }
 
+// (Re)allocate the per-tile count rows and flags for the context's current tile size.
+bool alloc_scan_scratch(moe_ctx *ctx, cudaStream_t st)
+{
+    const Derived &d = ctx->d;
+    const size_t tiles = ((size_t)ctx->cfg.max_tokens + d.tokens_per_block - 1) / d.tokens_per_block;
+    if (tiles > ctx->scan_tiles) {
+        cudaFree(ctx->d_tile_counts); cudaFree(ctx->d_tile_flag);
+        ctx->d_tile_counts = nullptr; ctx->d_tile_flag = nullptr; ctx->scan_tiles = 0;
+        if (cudaMalloc(&ctx->d_tile_counts, tiles * d.p_pad * sizeof(uint16_t)) != cudaSuccess ||
+            cudaMalloc(&ctx->d_tile_flag, tiles * sizeof(unsigned)) != cudaSuccess)
+            return false;
+        ctx->scan_tiles = tiles;
+    }
+    // flag 0 never equals an epoch (epochs start at 1 and skip 0)
+    return cudaMemsetAsync(ctx->d_tile_flag, 0, ctx->scan_tiles * sizeof(unsigned), st) == cudaSuccess;
+}
+
+// The kernels with rings in dynamic shared memory may use all of it.  The attribute belongs to
+// the function, not to a context, so it is set once per process to the largest size any
+// context can ask for.
+bool set_kernel_attributes_once()
+{
+    static std::once_flag once;
+    static bool ok = false;
+    std::call_once(once, [] {
+        const cudaFuncAttribute at = cudaFuncAttributeMaxDynamicSharedMemorySize;
+        const int sm = (int)(kMaxSmem - 1024);
+        ok = cudaFuncSetAttribute(k_scatter_bulk, at, sm) == cudaSuccess
+          && cudaFuncSetAttribute(k_combine_bulk<1, 8>, at, sm) == cudaSuccess
+          && cudaFuncSetAttribute(k_combine_bulk<2, 8>, at, sm) == cudaSuccess
+          && cudaFuncSetAttribute(k_combine_bulk<4, 8>, at, sm) == cudaSuccess
+          && cudaFuncSetAttribute(k_combine_bulk<1, 2>, at, sm) == cudaSuccess
+          && cudaFuncSetAttribute(k_combine_bulk<2, 2>, at, sm) == cudaSuccess
+          && cudaFuncSetAttribute(k_combine_bulk<4, 2>, at, sm) == cudaSuccess
+          && cudaFuncSetAttribute(k_combine_bulk<1, 0>, at, sm) == cudaSuccess
+          && cudaFuncSetAttribute(k_combine_bulk<2, 0>, at, sm) == cudaSuccess
+          && cudaFuncSetAttribute(k_combine_bulk<4, 0>, at, sm) == cudaSuccess;
+    });
+    return ok;
+}
+
+int tuned(const moe_ctx *ctx, int option, int dflt)
+{
+    return ctx->tune[option] >= 0 ? ctx->tune[option] : dflt;
+}
+
+// Launch shapes of the three kernels from the context's shape and its tuning overrides.
+void configure_launch(moe_ctx *ctx)
+{
+    const Derived &d = ctx->d;
+    ctx->route_smem = route_smem_bytes(d.E, d.max_rep, d.tokens_per_block, d.k, d.P);
+    ctx->spin_limit = (unsigned)tuned(ctx, MOE_TUNE_SPIN_LIMIT, (int)kDefaultSpinLimit);
+    ctx->pdl = tuned(ctx, MOE_TUNE_PDL, 1) != 0;
+    ctx->scatter_impl = tuned(ctx, MOE_TUNE_SCATTER_IMPL, 0);
+    ctx->bulk_stages = std::min(8, std::max(1, tuned(ctx, MOE_TUNE_SCATTER_BULK_STAGES, 4)));
+    const size_t stage_bytes = ((size_t)d.H * 2 + 127) & ~(size_t)127;
+    while (ctx->bulk_stages > 1 && ctx->bulk_stages * stage_bytes > kMaxSmem - 2048) --ctx->bulk_stages;
+    if (ctx->bulk_stages * stage_bytes > kMaxSmem - 2048) ctx->scatter_impl = 0;   // row too wide to stage
+    const size_t ring = ctx->bulk_stages * stage_bytes;
+    const int fit = std::max(1, (int)((kMaxSmem - 1024) / (ring + 1024)));
+    ctx->bulk_ctas_per_sm = std::min(fit, std::min(32, std::max(1, tuned(ctx, MOE_TUNE_SCATTER_BULK_CTAS_PER_SM, fit))));
+    ctx->scatter_blocks_per_sm = std::max(1, tuned(ctx, MOE_TUNE_SCATTER_BLOCKS_PER_SM, 8));
+    // one warp moves a whole row when it fits (long contiguous HBM bursts per destination
+    // row measured 6.3 TB/s against 5.65 TB/s with 2 KB pieces): 16-byte units per lane
+    {
+        static const int kUnroll[] = {4, 8, 16, 28, 32};
+        const int need = (d.H / 8 + 31) / 32;
+        int un = 32;
+        for (int u : kUnroll) if (u >= need) { un = u; break; }
+        const int forced = tuned(ctx, MOE_TUNE_SCATTER_UNROLL, 0);
+        for (int u : kUnroll) if (u == forced) un = forced;
+        ctx->scatter_unroll = un;
+    }
+    ctx->combine_blocks_per_sm = 8;
+    ctx->combine_impl = tuned(ctx, MOE_TUNE_COMBINE_IMPL, 1);
+    // a ring stage holds one column chunk of all k rows: widen the chunk for small k so that a
+    // stage stays near 4 KB and the ring keeps as many bytes in flight as with k = 8
+    int u_auto = d.k <= 2 ? 4 : (d.k <= 4 ? 2 : 1);
+    while (u_auto > 1 && 32 * u_auto > d.H / 8) u_auto /= 2;        // never wider than a row
+    ctx->combine_u = tuned(ctx, MOE_TUNE_COMBINE_CHUNK, u_auto);
+    if (ctx->combine_u != 1 && ctx->combine_u != 2 && ctx->combine_u != 4) ctx->combine_u = 2;
+    // ring shape: with many rows per token (k >= 6) four warps per CTA with five stages each
+    // (two CTAs per SM: 8 warps, ~160 KB of rings) measured 4-7 % faster than eight warps with
+    // three stages; with few rows per token the wider, shallower shape is the faster one
+    const bool deep = d.k >= 6;
+    ctx->combine_warps = std::min(kCombineBulkMaxWarps, std::max(1, tuned(ctx, MOE_TUNE_COMBINE_WARPS, deep ? 4 : 8)));
+    ctx->combine_stages = std::min(8, std::max(2, tuned(ctx, MOE_TUNE_COMBINE_STAGES, deep ? 5 : 3)));
+    while (ctx->combine_stages > 2 &&
+           combine_bulk_smem(ctx->combine_stages, d.k, ctx->combine_u, ctx->combine_warps) > kMaxSmem - 1024)
+        --ctx->combine_stages;
+    ctx->combine_smem = combine_bulk_smem(ctx->combine_stages, d.k, ctx->combine_u, ctx->combine_warps);
+    if (ctx->combine_smem > kMaxSmem - 1024) ctx->combine_impl = 0;
+    const int fit_c = std::max(1, (int)((kMaxSmem - 1024) / (ctx->combine_smem + 1024)));
+    ctx->combine_ctas_per_sm = std::max(1, std::min(fit_c, tuned(ctx, MOE_TUNE_COMBINE_CTAS_PER_SM, fit_c)));
+}
+
 void free_ctx(moe_ctx *ctx)
 {
     if (!ctx) return;
-    cudaFree(ctx->d_state); cudaFree(ctx->d_bias); cudaFree(ctx->d_slot_scale);
-    cudaFree(ctx->d_desc); cudaFree(ctx->d_ctl); cudaFree(ctx->d_pos);
+    cudaFree(ctx->d_state); cudaFree(ctx->d_live); cudaFree(ctx->d_bias); cudaFree(ctx->d_slot_scale);
+    cudaFree(ctx->d_tile_counts); cudaFree(ctx->d_tile_flag); cudaFree(ctx->d_ctl); cudaFree(ctx->d_pos);
+    cudaFree(ctx->d_zero_row);
     cudaFree(ctx->d_peer_bufs); cudaFree(ctx->d_src_base);
     for (int s = 0; s < kStagingSlots; ++s) {
         if (ctx->h_stage[s]) cudaFreeHost(ctx->h_stage[s]);
@@ -499,19 +621,22 @@ moe_status moe_route_init(const moe_config *cfg, const int32_t *slot_to_expert, 
     for (int s = 0; s < kStagingSlots; ++s) {
         ctx->h_stage[s] = nullptr; ctx->stage_done[s] = nullptr; ctx->stage_used[s] = false;
     }
-    ctx->d_state = nullptr; ctx->d_bias = nullptr; ctx->d_slot_scale = nullptr;
-    ctx->d_desc = nullptr; ctx->d_ctl = nullptr; ctx->d_pos = nullptr;
+    ctx->d_state = nullptr; ctx->d_live = nullptr; ctx->d_bias = nullptr; ctx->d_slot_scale = nullptr;
+    ctx->d_tile_counts = nullptr; ctx->d_tile_flag = nullptr; ctx->scan_tiles = 0;
+    ctx->d_ctl = nullptr; ctx->d_pos = nullptr; ctx->d_zero_row = nullptr;
+    for (int i = 0; i < kNumTuning; ++i) ctx->tune[i] = -1;
 
     bool ok = cudaGetDevice(&ctx->device) == cudaSuccess &&
               cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device) ==
                   cudaSuccess;
-    const size_t tiles = ((size_t)cfg->max_tokens + d.tokens_per_block - 1) / d.tokens_per_block;
     ok = ok && cudaMalloc(&ctx->d_state, (size_t)d.state_words * 4) == cudaSuccess;
+    ok = ok && cudaMalloc(&ctx->d_live, (size_t)d.E * (1 + d.max_rep) * 4) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->d_bias, (size_t)d.E * 4) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->d_slot_scale, (size_t)d.P * 4) == cudaSuccess;
-    ok = ok && cudaMalloc(&ctx->d_desc, tiles * d.P * sizeof(unsigned long long)) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->d_ctl, sizeof(moe::Control)) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->d_pos, (size_t)cfg->max_tokens * d.k * 4) == cudaSuccess;
+    ok = ok && cudaMalloc(&ctx->d_zero_row, (size_t)d.H * 2) == cudaSuccess;
+    ok = ok && alloc_scan_scratch(ctx, st);
     for (int s = 0; s < kStagingSlots && ok; ++s) {
         ok = cudaMallocHost(&ctx->h_stage[s], (size_t)d.state_words * 4) == cudaSuccess &&
              cudaEventCreateWithFlags(&ctx->stage_done[s], cudaEventDisableTiming) == cudaSuccess;
@@ -522,75 +647,16 @@ moe_status moe_route_init(const moe_config *cfg, const int32_t *slot_to_expert, 
         if (bias) std::copy(bias, bias + d.E, b.begin());
         const moe::Control c0 = {0u, 1u, kDevOk, 0};
         // synchronous pageable copies: the host arrays may be freed on return
-        ok = cudaMemsetAsync(ctx->d_desc, 0, tiles * d.P * sizeof(unsigned long long), st) == cudaSuccess &&
+        ok = cudaMemsetAsync(ctx->d_zero_row, 0, (size_t)d.H * 2, st) == cudaSuccess &&
              cudaMemcpyAsync(ctx->d_ctl, &c0, sizeof(c0), cudaMemcpyHostToDevice, st) == cudaSuccess &&
              cudaMemcpyAsync(ctx->d_bias, b.data(), (size_t)d.E * 4, cudaMemcpyHostToDevice, st) == cudaSuccess &&
              cudaMemcpyAsync(ctx->d_slot_scale, slot_scale, (size_t)d.P * 4, cudaMemcpyHostToDevice, st) == cudaSuccess &&
              cudaMemcpyAsync(ctx->d_state, blob.data(), (size_t)d.state_words * 4, cudaMemcpyHostToDevice, st) == cudaSuccess &&
+             enqueue_derive(ctx, st) == MOE_OK &&
              cudaStreamSynchronize(st) == cudaSuccess;
     }
-    if (ok) {
-        ctx->route_smem = route_smem_bytes(d.E, d.max_rep, d.tokens_per_block, d.k, d.P);
-        ctx->pdl = env_int("MOE_PDL", 1) != 0;
-        ctx->scatter_impl = env_int("MOE_SCATTER_IMPL", 0);
-        ctx->bulk_stages = std::min(8, std::max(1, env_int("MOE_BULK_STAGES", 4)));
-        const size_t stage_bytes = ((size_t)d.H * 2 + 127) & ~(size_t)127;
-        while (ctx->bulk_stages > 1 && ctx->bulk_stages * stage_bytes > kMaxSmem - 2048) --ctx->bulk_stages;
-        if (ctx->bulk_stages * stage_bytes > kMaxSmem - 2048) ctx->scatter_impl = 0;   // row too wide to stage
-        const size_t ring = ctx->bulk_stages * stage_bytes;
-        int fit = (int)((kMaxSmem - 1024) / (ring + 1024));
-        ctx->bulk_ctas_per_sm = std::min(32, std::max(1, env_int("MOE_BULK_CTAS_PER_SM", fit)));
-        if (ctx->bulk_ctas_per_sm > fit) ctx->bulk_ctas_per_sm = std::max(1, fit);
-        if (ctx->scatter_impl == 1)
-            ok = cudaFuncSetAttribute(k_scatter_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      (int)ring) == cudaSuccess;
-        ctx->scatter_blocks_per_sm = std::max(1, env_int("MOE_SCATTER_BLOCKS_PER_SM", 8));
-        // one warp moves a whole row when it fits (long contiguous HBM bursts per destination
-        // row measured 6.3 TB/s against 5.65 TB/s with 2 KB pieces): 16-byte units per lane
-        {
-            static const int kUnroll[] = {4, 8, 16, 28, 32};
-            const int need = (d.H / 8 + 31) / 32;
-            int un = 32;
-            for (int u : kUnroll) if (u >= need) { un = u; break; }
-            const int forced = env_int("MOE_SCATTER_UNROLL", 0);
-            for (int u : kUnroll) if (u == forced) un = forced;
-            ctx->scatter_unroll = un;
-        }
-        ctx->combine_blocks_per_sm = std::max(1, env_int("MOE_COMBINE_BLOCKS_PER_SM", 8));
-        ctx->combine_impl = env_int("MOE_COMBINE_IMPL", 1);
-        // a ring stage holds one column chunk of all k rows: widen the chunk for small k so that a
-        // stage stays near 4 KB and the ring keeps as many bytes in flight as with k = 8
-        int u_auto = d.k <= 2 ? 4 : (d.k <= 4 ? 2 : 1);
-        while (u_auto > 1 && 32 * u_auto > d.H / 8) u_auto /= 2;        // never wider than a row
-        ctx->combine_u = env_int("MOE_COMBINE_U", u_auto);
-        if (ctx->combine_u != 1 && ctx->combine_u != 2 && ctx->combine_u != 4) ctx->combine_u = 2;
-        // ring shape: with many rows per token (k >= 6) four warps per CTA with five stages each
-        // (two CTAs per SM: 8 warps, ~160 KB of rings) measured 4-7 % faster than eight warps with
-        // three stages; with few rows per token the wider, shallower shape is the faster one
-        const bool deep = d.k >= 6;
-        ctx->combine_warps = std::min(kCombineBulkMaxWarps, std::max(1, env_int("MOE_COMBINE_WARPS", deep ? 4 : 8)));
-        ctx->combine_stages = std::min(8, std::max(2, env_int("MOE_COMBINE_STAGES", deep ? 5 : 3)));
-        while (ctx->combine_stages > 2 &&
-               combine_bulk_smem(ctx->combine_stages, d.k, ctx->combine_u, ctx->combine_warps) > kMaxSmem - 1024)
-            --ctx->combine_stages;
-        ctx->combine_smem = combine_bulk_smem(ctx->combine_stages, d.k, ctx->combine_u, ctx->combine_warps);
-        if (ctx->combine_smem > kMaxSmem - 1024) ctx->combine_impl = 0;
-        if (ctx->combine_impl == 1) {
-            const int fit_c = (int)((kMaxSmem - 1024) / (ctx->combine_smem + 1024));
-            ctx->combine_ctas_per_sm = std::max(1, std::min(fit_c, env_int("MOE_COMBINE_CTAS_PER_SM", fit_c)));
-            const int sm = (int)ctx->combine_smem;
-            const cudaFuncAttribute at = cudaFuncAttributeMaxDynamicSharedMemorySize;
-            ok = ok && cudaFuncSetAttribute(k_combine_bulk<1, 8>, at, sm) == cudaSuccess
-                    && cudaFuncSetAttribute(k_combine_bulk<2, 8>, at, sm) == cudaSuccess
-                    && cudaFuncSetAttribute(k_combine_bulk<4, 8>, at, sm) == cudaSuccess
-                    && cudaFuncSetAttribute(k_combine_bulk<1, 2>, at, sm) == cudaSuccess
-                    && cudaFuncSetAttribute(k_combine_bulk<2, 2>, at, sm) == cudaSuccess
-                    && cudaFuncSetAttribute(k_combine_bulk<4, 2>, at, sm) == cudaSuccess
-                    && cudaFuncSetAttribute(k_combine_bulk<1, 0>, at, sm) == cudaSuccess
-                    && cudaFuncSetAttribute(k_combine_bulk<2, 0>, at, sm) == cudaSuccess
-                    && cudaFuncSetAttribute(k_combine_bulk<4, 0>, at, sm) == cudaSuccess;
-        }
-    }
+    ok = ok && set_kernel_attributes_once();
+    if (ok) configure_launch(ctx);
     if (!ok) {
         cudaGetLastError();
         free_ctx(ctx);
@@ -740,7 +806,7 @@ moe_status moe_dispatch(moe_ctx *ctx, const float *logits, const void *x, int32_
 
     ScatterParams sp;
     sp.x = static_cast<const uint4 *>(x); sp.send = static_cast<uint4 *>(out->send_buf);
-    sp.T = T; sp.k = d.k; sp.hv = d.H / 8;
+    sp.T = T; sp.k = d.k; sp.hv = d.H / 8; sp.P = d.P; sp.spin_limit = ctx->spin_limit;
     sp.topk_slot = out->topk_slot; sp.slot_offsets = out->slot_offsets; sp.pos_in_slot = ctx->d_pos;
     sp.dst_row = out->dst_row; sp.src_index = out->src_index; sp.ctl = ctx->d_ctl;
     if (ctx->scatter_impl == 1) {
@@ -780,6 +846,7 @@ moe_status moe_combine(moe_ctx *ctx, const void *expert_buf, int32_t T, void *y,
     cp.dst_row = ctx->last_dst_row; cp.topk_weights = ctx->last_weights; cp.topk_slot = ctx->last_slot;
     cp.slot_scale = ctx->d_slot_scale;
     cp.peer_bufs = nullptr; cp.slots_per_gpu = 0;
+    cp.P = d.P; cp.row_limit = (long long)T * d.k; cp.zero_row = ctx->d_zero_row; cp.spin_limit = ctx->spin_limit;
     if (ctx->combine_impl == 1) return enqueue_combine_bulk(ctx, cp, st);
     const int chunks = (cp.hv + kCombineChunk - 1) / kCombineChunk;
     const long long items = (long long)T * chunks;
@@ -893,7 +960,7 @@ moe_status moe_ep_scatter(moe_ctx *ctx, const void *x, int32_t T, const int32_t 
     if (T == 0) return MOE_OK;
     EpScatterParams sp;
     sp.x = static_cast<const uint4 *>(x); sp.peer_bufs = ctx->d_peer_bufs;
-    sp.T = T; sp.k = d.k; sp.hv = d.H / 8; sp.spg = ctx->ep_spg; sp.recv_rows = ctx->ep_recv_rows;
+    sp.T = T; sp.k = d.k; sp.hv = d.H / 8; sp.spg = ctx->ep_spg; sp.P = d.P; sp.recv_rows = ctx->ep_recv_rows;
     sp.topk_slot = ctx->last_slot; sp.src_base = ctx->d_src_base; sp.pos_in_slot = ctx->d_pos;
     sp.dst_row = const_cast<int32_t *>(ctx->last_dst_row);
     const int un = ctx->scatter_unroll;
@@ -925,6 +992,7 @@ moe_status moe_ep_combine(moe_ctx *ctx, int32_t T, void *y, void *cuda_stream)
     cp.dst_row = ctx->last_dst_row; cp.topk_weights = ctx->last_weights; cp.topk_slot = ctx->last_slot;
     cp.slot_scale = ctx->d_slot_scale;
     cp.peer_bufs = const_cast<const uint4 *const *>(ctx->d_peer_bufs); cp.slots_per_gpu = ctx->ep_spg;
+    cp.P = d.P; cp.row_limit = ctx->ep_recv_rows; cp.zero_row = ctx->d_zero_row; cp.spin_limit = ctx->spin_limit;
     return enqueue_combine_bulk(ctx, cp, st);
 }
 
@@ -960,6 +1028,48 @@ moe_status moe_step_host(moe_ctx *ctx, const float *logits_host, const void *x_h
                                               y_host, cuda_stream);
     if (ms != MOE_OK) return ms;
     return cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+moe_status moe_set_tuning(moe_ctx *ctx, int32_t option, int32_t value)
+{
+    if (!ctx || option < 0 || option >= kNumTuning || value < -1) return MOE_ERR_INVALID_ARG;
+    if (cudaDeviceSynchronize() != cudaSuccess) return MOE_ERR_CUDA;
+    const int before = ctx->tune[option];
+    ctx->tune[option] = value;
+    if (option == MOE_TUNE_ROUTE_LANES_PER_TOKEN || option == MOE_TUNE_ROUTE_TOKENS_PER_TILE) {
+        // the routing tile decides the size of the scan scratch: derive again and regrow it
+        Derived d;
+        if (!derive(&ctx->cfg, &d, std::max(0, ctx->tune[MOE_TUNE_ROUTE_LANES_PER_TOKEN]),
+                    std::max(0, ctx->tune[MOE_TUNE_ROUTE_TOKENS_PER_TILE]))) {
+            ctx->tune[option] = before;
+            return MOE_ERR_INVALID_ARG;
+        }
+        const Derived old = ctx->d;
+        ctx->d = d;
+        if (!alloc_scan_scratch(ctx, nullptr) || cudaDeviceSynchronize() != cudaSuccess) {
+            cudaGetLastError();
+            ctx->d = old; ctx->tune[option] = before;
+            return MOE_ERR_CUDA;
+        }
+        ctx->device_bytes = device_bytes_for(d, ctx->cfg.max_tokens);
+    }
+    configure_launch(ctx);
+    if (option == MOE_TUNE_COMBINE_IMPL && ctx->ep_world > 0 && ctx->combine_impl != 1) {
+        ctx->tune[option] = before;                        // the group mode needs the ring combine
+        configure_launch(ctx);
+        return MOE_ERR_INVALID_ARG;
+    }
+    return MOE_OK;
+}
+
+moe_status moe_debug_skip_ticket(moe_ctx *ctx)
+{
+    if (!ctx) return MOE_ERR_INVALID_ARG;
+    const unsigned one = 1u;
+    if (cudaDeviceSynchronize() != cudaSuccess ||
+        cudaMemcpy(&ctx->d_ctl->ticket, &one, sizeof(one), cudaMemcpyHostToDevice) != cudaSuccess)
+        return MOE_ERR_CUDA;
+    return MOE_OK;
 }
 
 moe_status moe_set_timing_event(moe_ctx *ctx, void *cuda_event)

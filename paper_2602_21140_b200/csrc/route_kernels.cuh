@@ -11,12 +11,13 @@
 // lane busy in the serial top-k rounds (the kernel is bound by instruction
 // issue, not by memory).
 //
-// Prefix over tiles: the whole problem fits in one wave of CTAs, so all tiles
-// publish at about the same time and a chained look-back (wait for the
-// predecessor's inclusive prefix) would serialise them.  Instead every tile
-// publishes only its own per-slot aggregate and sums the aggregates of ALL
-// earlier tiles with independent, coalesced loads; the host keeps the number
-// of tiles <= 128 by growing the tile with max_tokens, which bounds that traffic.
+// Prefix over tiles: the whole problem fits in one wave of CTAs (the host sizes the
+// tile so that a step has about one tile per SM), so all tiles publish at about the
+// same time and a chained look-back (wait for the predecessor's inclusive prefix)
+// would serialise them.  Instead every tile publishes only its own per-slot counts
+// (16-bit, eight to a 16-byte store) followed by one flag word carrying the step's
+// epoch, waits for the flags of ALL earlier tiles (one polling thread per tile) and
+// sums their counts with independent 16-byte loads: two L2 round trips in all.
 #pragma once
 
 #include "device_utils.cuh"
@@ -35,9 +36,40 @@ constexpr int kRouteWarps = kRouteThreads / 32;
 //                        layout (logical-rank order; identity unless ranks were compacted)
 constexpr int kStateHeaderWords = 2;
 
-// Look-back descriptor, one 64-bit word per (tile, slot):
-//   bits 63..32 epoch of the step that wrote it, 31..0 assignments of the tile on the slot
-constexpr int kMaxRouteTiles = 128;
+// A step has at most this many tiles (one polling thread per earlier tile in the look-back).
+constexpr int kMaxRouteTiles = kRouteThreads;
+
+// Live-replica lists derived from the state blob: per expert 1 + max_rep words, the number of
+// live replicas followed by their slots in ascending order.  k_derive_live rebuilds them on
+// the stream right after every state copy, so the routing kernel loads one flat table
+// instead of chasing bitmap words through the replica table in every CTA of every step.
+struct DeriveParams {
+    const int32_t *state;
+    int E, S, max_rep, rank_words, expert_words;
+    int32_t *live;            // out [E][1 + max_rep]
+};
+
+constexpr int kDeriveThreads = 256;
+
+__global__ void __launch_bounds__(kDeriveThreads) k_derive_live(DeriveParams p)
+{
+    const uint32_t *alive = reinterpret_cast<const uint32_t *>(p.state + kStateHeaderWords);
+    const uint32_t *lost = alive + p.rank_words;
+    const int32_t *table = p.state + kStateHeaderWords + p.rank_words + p.expert_words;
+    const int e = blockIdx.x * kDeriveThreads + threadIdx.x;
+    if (e >= p.E) return;
+    int32_t *ent = p.live + (size_t)e * (1 + p.max_rep);
+    const bool expert_ok = !((lost[e >> 5] >> (e & 31)) & 1u);
+    int n = 0;
+    for (int r = 0; r < p.max_rep; ++r) {
+        const int slot = table[e * p.max_rep + r];         // ascending, -1 padded
+        ent[1 + r] = -1;
+        if (slot < 0 || !expert_ok) continue;
+        const int rank = slot / p.S;
+        if ((alive[rank >> 5] >> (rank & 31)) & 1u) ent[1 + n++] = slot;
+    }
+    ent[0] = n;
+}
 
 struct RouteParams {
     const float *logits;      // [T,E]
@@ -45,22 +77,27 @@ struct RouteParams {
     int score_func, n_group, topk_group, lanes_per_group, group_m;
     float route_scale;
     int tokens_per_block;
+    int p_pad;                // P rounded up to a multiple of 8: row pitch of tile_counts
     int rank_words, expert_words;
-    const int32_t *state;     // routing state blob
+    unsigned spin_limit;      // polls before a bounded wait gives up
+    const int32_t *state;     // routing state blob (header and slot order are read here)
+    const int32_t *live;      // derived live-replica lists [E][1 + max_rep]
     const float *bias;        // [E]
     int32_t *topk_ids;        // [T,k]
     float *topk_weights;      // [T,k]
     int32_t *topk_slot;       // [T,k]
     int32_t *pos_in_slot;     // [T*k]: stable rank of assignment i inside its slot
     int32_t *slot_counts, *slot_offsets, *rank_counts, *rank_offsets;
-    unsigned long long *desc; // [tiles, P]
+    uint16_t *tile_counts;    // [tiles][p_pad]: assignments of each tile on each slot
+    unsigned *tile_flag;      // [tiles]: epoch of the step whose counts the row holds
     Control *ctl;
 };
 
 __host__ __device__ inline size_t route_smem_bytes(int E, int max_rep, int tokens_per_block, int k,
                                                    int P)
 {
-    size_t words = (size_t)E + (size_t)E * max_rep + 2 * (size_t)tokens_per_block * k + 3 * (size_t)P;
+    const size_t p_pad = ((size_t)P + 7) & ~(size_t)7;
+    size_t words = (size_t)E * (1 + max_rep) + 2 * (size_t)tokens_per_block * k + 2 * p_pad + (size_t)P;
     return words * sizeof(int32_t) + (size_t)kRouteWarps * P * sizeof(uint16_t);
 }
 
@@ -90,9 +127,8 @@ __device__ __forceinline__ void rescan_block(uint32_t (&code)[EPL], uint32_t (&b
 // expert, the weight and the physical slot.
 template <int EPL, int LPT>
 __device__ __forceinline__ void route_tokens(const RouteParams &p, int t_first, uint32_t avail_mask,
-                                             const int32_t *s_nlive, const int32_t *s_live,
-                                             int fallback_expert, int &out_id, float &out_w,
-                                             int &out_slot)
+                                             const int32_t *s_live, int fallback_expert, int &out_id,
+                                             float &out_w, int &out_slot)
 {
     const unsigned full = 0xffffffffu;
     const int lane = lane_id();
@@ -105,7 +141,7 @@ __device__ __forceinline__ void route_tokens(const RouteParams &p, int t_first, 
     const bool sigmoid = p.score_func != 0;
     const bool grouped = p.n_group > 1;
 
-    // a1 gate scores, a2 availability mask, and the two best keys of this lane (for a3)
+    // gate scores, availability mask, and the two best keys of this lane (for the group scores)
     uint32_t code[EPL];
     float h1 = neg_inf, h2 = neg_inf;
 #pragma unroll
@@ -137,7 +173,7 @@ __device__ __forceinline__ void route_tokens(const RouteParams &p, int t_first, 
         }
     }
 
-    // a3 group-limited selection: score = sum of the (up to) group_m best finite keys
+    // group-limited selection: score = sum of the (up to) group_m best finite keys
     bool active = true;
     if (p.n_group > 1) {
         for (int off = 1; off < p.lanes_per_group; off <<= 1) {
@@ -157,7 +193,7 @@ __device__ __forceinline__ void route_tokens(const RouteParams &p, int t_first, 
         active = (g < p.n_group) && (rank < p.topk_group);
     }
 
-    // a4 top-k: k rounds of arg-max over order-preserving integer codes.  A lane keeps the best
+    // top-k: k rounds of arg-max over order-preserving integer codes.  A lane keeps the best
     // code of each block of four of its experts, so that after a pick only the block that lost
     // an element is scanned again (the rounds are bound by instruction issue).
     constexpr int kBlocks = (EPL + 3) / 4;
@@ -203,7 +239,7 @@ __device__ __forceinline__ void route_tokens(const RouteParams &p, int t_first, 
         }
     }
 
-    // a5 weights: ratio of the chosen scores, summed and divided in double.  The score of a
+    // weights: ratio of the chosen scores, summed and divided in double.  The score of a
     // chosen expert is recomputed from its logit (same operations, same bits as above).
     float my_val = 0.0f;
     if (sl < p.k) {
@@ -221,12 +257,12 @@ __device__ __forceinline__ void route_tokens(const RouteParams &p, int t_first, 
     for (int j = 0; j < p.k; ++j) usum += __shfl_sync(full, u, j, LPT);
     out_w = (float)((double)p.route_scale * u / usum);
 
-    // a6 replica pick: (t mod live count)-th entry of the ascending live list
+    // replica pick: (t mod live count)-th entry of the ascending live list
     out_id = my_id;
     out_slot = -1;
     if (sl < p.k) {
-        const int n = s_nlive[my_id];
-        out_slot = s_live[my_id * p.max_rep + (t % n)];
+        const int32_t *ent = s_live + my_id * (1 + p.max_rep);
+        out_slot = ent[1 + t % ent[0]];
     }
     if (__any_sync(full, my_bad) && lane == 0) report_status(p.ctl, kDevInsufficientExperts);
 }
@@ -237,19 +273,23 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
     extern __shared__ int32_t smem[];
     const int E = p.E, P = p.P, k = p.k, tb = p.tokens_per_block;
     const int NA = tb * k;
-    int32_t *s_nlive = smem;                          // [E]
-    int32_t *s_live = s_nlive + E;                    // [E][max_rep]
-    int32_t *s_slot = s_live + E * p.max_rep;         // [NA] slot of each assignment of the tile
+    const int live_words = 1 + p.max_rep;
+    int32_t *s_live = smem;                           // [E][1 + max_rep] live count, live slots
+    int32_t *s_slot = s_live + E * live_words;        // [NA] slot of each assignment of the tile
     int32_t *s_lrank = s_slot + NA;                   // [NA] stable rank inside the tile
-    int32_t *s_hist = s_lrank + NA;                   // [P]  tile histogram (running)
-    int32_t *s_excl = s_hist + P;                     // [P]  assignments on slot p in earlier tiles
-    int32_t *s_order = s_excl + P;                    // [P]  physical slot at each layout position
+    int32_t *s_hist = s_lrank + NA;                   // [p_pad] tile histogram (running)
+    int32_t *s_excl = s_hist + p.p_pad;               // [p_pad] assignments on slot p in earlier tiles
+    int32_t *s_order = s_excl + p.p_pad;              // [P]  physical slot at each layout position
     uint16_t *s_wcount = reinterpret_cast<uint16_t *>(s_order + P);  // [32][P] one round's counts
     __shared__ unsigned s_ticket, s_epoch;
     __shared__ int s_warp_sums[kRouteWarps];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned full = 0xffffffffu;
+
+    // Before the wait only this CTA's own shared memory is touched.
+    for (int q = tid; q < p.p_pad; q += kRouteThreads) { s_hist[q] = 0; s_excl[q] = 0; }
+    for (int q = tid; q < kRouteWarps * P; q += kRouteThreads) s_wcount[q] = 0;
 
     // Wait for the previous kernel first and only then let the scatter be scheduled: the scatter
     // requests its first x rows before its own wait, which is safe only once whatever produced x
@@ -263,38 +303,21 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
         s_ticket = (unsigned)te;
         s_epoch = (unsigned)(te >> 32);
     }
-    // Live replica lists from the rank bitmap and the replica table (a2, a6).
-    const uint32_t *alive = reinterpret_cast<const uint32_t *>(p.state + kStateHeaderWords);
-    const uint32_t *lost = alive + p.rank_words;
-    const int32_t *table = p.state + kStateHeaderWords + p.rank_words + p.expert_words;
-    for (int e = tid; e < E; e += kRouteThreads) {
-        // first every replica slot of the expert, then the alive words they point to: two
-        // rounds of independent loads instead of a chain through the replicas
-        constexpr int kMaxRep = 8;
-        int slot[kMaxRep];
-        uint32_t word[kMaxRep];
-        const uint32_t lost_word = lost[e >> 5];
-#pragma unroll
-        for (int r = 0; r < kMaxRep; ++r) slot[r] = (r < p.max_rep) ? table[e * p.max_rep + r] : -1;
-#pragma unroll
-        for (int r = 0; r < kMaxRep; ++r) word[r] = (slot[r] >= 0) ? alive[(slot[r] / p.S) >> 5] : 0u;
-        const bool expert_ok = !((lost_word >> (e & 31)) & 1u);
-        int n = 0;
-#pragma unroll
-        for (int r = 0; r < kMaxRep; ++r)
-            if (expert_ok && slot[r] >= 0 && ((word[r] >> ((slot[r] / p.S) & 31)) & 1u))
-                s_live[e * p.max_rep + n++] = slot[r];
-        s_nlive[e] = n;
-    }
-    // layout order of the slots, for the final scan of the last tile
+    // live replica lists (availability mask and replica pick) and the layout order of the slots
+    for (int i = tid; i < E * live_words; i += kRouteThreads) s_live[i] = p.live[i];
     const int32_t *order = p.state + kStateHeaderWords + p.rank_words + p.expert_words + E * p.max_rep;
-    for (int q = tid; q < P; q += kRouteThreads) { s_hist[q] = 0; s_excl[q] = 0; s_order[q] = order[q]; }
-    for (int q = tid; q < kRouteWarps * P; q += kRouteThreads) s_wcount[q] = 0;
+    for (int q = tid; q < P; q += kRouteThreads) s_order[q] = order[q];
     const int fallback_expert = p.state[0];
     __syncthreads();
 
     const unsigned ticket = s_ticket;
-    const unsigned long long epoch = s_epoch;
+    const unsigned epoch = s_epoch;
+    if (ticket >= gridDim.x) {
+        // The control word was not armed for this step (an earlier step gave up and the host has
+        // not yet read the status): route nothing rather than index past the tile arrays.
+        if (tid == 0) report_status(p.ctl, kDevTimeout);
+        return;
+    }
     const int t0 = (int)ticket * tb;
     const int n_tok = min(tb, p.T - t0);
 
@@ -305,7 +328,7 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
 #pragma unroll
     for (int q = 0; q < EPL; ++q) {
         const int e = sl * EPL + q;
-        if (e < E && s_nlive[e] > 0) avail_mask |= 1u << q;
+        if (e < E && s_live[e * live_words] > 0) avail_mask |= 1u << q;
     }
 
     // Dense-FFN mode (score_func 2): the "experts" are the k = TP shards of E/k replicated
@@ -316,7 +339,7 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
             int n = 0;
             for (int g = 0; g < E / k; ++g) {
                 bool healthy = true;
-                for (int sh = 0; sh < k; ++sh) healthy = healthy && (s_nlive[g * k + sh] > 0);
+                for (int sh = 0; sh < k; ++sh) healthy = healthy && (s_live[(g * k + sh) * live_words] > 0);
                 if (healthy) s_lrank[n++] = g;             // s_lrank is free until the histogram step
             }
             s_warp_sums[0] = n;
@@ -325,7 +348,7 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
     }
     const int n_healthy = dense ? s_warp_sums[0] : 0;
 
-    // ---- a1..a6 per token -------------------------------------------------
+    // ---- gate, mask, selection, weights, replica: per token ----------------
     for (int lt0 = warp * kTokPerWarp; lt0 < tb; lt0 += kRouteWarps * kTokPerWarp) {
         const int lt = lt0 + sub;
         const int t = t0 + lt;
@@ -337,10 +360,10 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
                 if (sl < k && t < p.T) {
                     id = s_lrank[t % n_healthy] * k + sl;
                     w = p.route_scale;
-                    slot = s_live[id * p.max_rep + (t % s_nlive[id])];
+                    slot = s_live[id * live_words + 1 + t % s_live[id * live_words]];
                 }
             } else {
-                route_tokens<EPL, LPT>(p, t0 + lt0, avail_mask, s_nlive, s_live, fallback_expert, id, w, slot);
+                route_tokens<EPL, LPT>(p, t0 + lt0, avail_mask, s_live, fallback_expert, id, w, slot);
             }
             if (t >= p.T) slot = -1;
             if (sl < k && t < p.T) {
@@ -354,7 +377,7 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
     }
     __syncthreads();
 
-    // ---- a7/a9 tile histogram and stable rank inside the tile --------------
+    // ---- tile histogram and stable rank of every assignment inside the tile 
     // Rounds of 1024 assignments in ascending i.  Inside a round, match_any gives
     // the rank among equal slots of a warp and the per-warp counts; a scan down
     // each slot's column of counts orders the warps.
@@ -384,47 +407,72 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
         }
     }
 
-    // ---- a8 prefix over tiles: publish this tile's aggregate, sum all earlier ones
-    for (int q = tid; q < P; q += kRouteThreads)
-        st_relaxed_u64(p.desc + (size_t)ticket * P + q, (epoch << 32) | (unsigned)s_hist[q]);
+    // ---- prefix over tiles: publish this tile's counts, sum those of all earlier tiles
+    {
+        uint4 *mine = reinterpret_cast<uint4 *>(p.tile_counts + (size_t)ticket * p.p_pad);
+        for (int q8 = tid; q8 < p.p_pad / 8; q8 += kRouteThreads) {
+            const int32_t *h = s_hist + 8 * q8;            // entries past P stay zero
+            uint4 v;
+            v.x = (unsigned)h[0] | ((unsigned)h[1] << 16); v.y = (unsigned)h[2] | ((unsigned)h[3] << 16);
+            v.z = (unsigned)h[4] | ((unsigned)h[5] << 16); v.w = (unsigned)h[6] | ((unsigned)h[7] << 16);
+            __stcg(mine + q8, v);
+        }
+    }
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();                                   // the counts of every thread, then the flag
+        st_relaxed_u32(p.tile_flag + ticket, epoch);
+    }
     if (ticket > 0) {
-        // thread = (segment g, slot q): segment g sums tiles g, g+nseg, ... of column q,
-        // eight independent loads at a time
-        constexpr int kBatch = 8;
-        const int nseg = max(1, min(32, kRouteThreads / P));
-        const int per_pass = max(1, kRouteThreads / nseg);        // slots handled per pass
+        // one thread per earlier tile waits for that tile's flag
         bool gave_up = false;
-        for (int q0 = 0; q0 < P; q0 += per_pass) {
-            const int g = tid / per_pass, q = q0 + tid % per_pass;
-            if (g >= nseg || q >= P) continue;
-            int partial = 0;
-            for (int b0 = g; b0 < (int)ticket && !gave_up; b0 += nseg * kBatch) {
-                unsigned long long v[kBatch];
+        if (tid < (int)ticket) {
+            unsigned spins = 0;
+            while (ld_acquire_u32(p.tile_flag + tid) != epoch) {
+                if (++spins > p.spin_limit ||
+                    ((spins & 255u) == 0 && ld_relaxed_s32(&p.ctl->status) == kDevTimeout)) {
+                    gave_up = true;
+                    break;
+                }
+                __nanosleep(kSpinSleepNs);
+            }
+        }
+        if (__syncthreads_or(gave_up)) {
+            // An earlier tile never published.  Nothing of this tile's placement is written, the
+            // control word stays as it is, and the status word tells the host (which re-arms it).
+            if (tid == 0) report_status(p.ctl, kDevTimeout);
+            return;
+        }
+        // thread = (segment g of the earlier tiles, group q8 of eight slots); every load is independent
+        const int groups = p.p_pad / 8;
+        const int nseg = kRouteThreads / groups;           // >= 2: P <= 4096
+        const int g = tid / groups, q8 = tid % groups;
+        if (g < nseg) {
+            constexpr int kBatch = 4;
+            int acc[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) acc[u] = 0;
+            for (int b0 = g; b0 < (int)ticket; b0 += nseg * kBatch) {
+                uint4 v[kBatch];
 #pragma unroll
                 for (int u = 0; u < kBatch; ++u) {
                     const int b = b0 + u * nseg;
-                    v[u] = (b < (int)ticket) ? ld_relaxed_u64(p.desc + (size_t)b * P + q) : (epoch << 32);
+                    v[u] = make_uint4(0u, 0u, 0u, 0u);
+                    if (b < (int)ticket)
+                        v[u] = __ldcg(reinterpret_cast<const uint4 *>(p.tile_counts + (size_t)b * p.p_pad) + q8);
                 }
 #pragma unroll
                 for (int u = 0; u < kBatch; ++u) {
-                    const int b = b0 + u * nseg;
-                    unsigned spins = 0;
-                    while ((v[u] >> 32) != epoch) {                // that tile has not published yet
-                        if (++spins > kSpinLimit ||
-                            ((spins & 1023u) == 0 && ld_relaxed_s32(&p.ctl->status) == kDevTimeout)) {
-                            gave_up = true;
-                            break;
-                        }
-                        __nanosleep(kSpinSleepNs);
-                        v[u] = ld_relaxed_u64(p.desc + (size_t)b * P + q);
-                    }
-                    if (gave_up) break;
-                    partial += (int)(unsigned)(v[u] & 0xFFFFFFFFull);
+                    acc[0] += v[u].x & 0xffffu; acc[1] += v[u].x >> 16;
+                    acc[2] += v[u].y & 0xffffu; acc[3] += v[u].y >> 16;
+                    acc[4] += v[u].z & 0xffffu; acc[5] += v[u].z >> 16;
+                    acc[6] += v[u].w & 0xffffu; acc[7] += v[u].w >> 16;
                 }
             }
-            if (partial) atomicAdd(&s_excl[q], partial);
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                if (acc[u]) atomicAdd(&s_excl[8 * q8 + u], acc[u]);
         }
-        if (gave_up) report_status(p.ctl, kDevTimeout);
     }
     __syncthreads();
 
@@ -434,7 +482,7 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
 
     if (ticket != gridDim.x - 1) return;
 
-    // ---- the last tile knows every total: a7 counts, a8 offsets -----------
+    // ---- the last tile knows every total: per-slot counts and offsets -----
     // exclusive scan over the P layout positions (position q holds physical slot order[q]),
     // a contiguous chunk of positions per thread
     for (int q = tid; q < P; q += kRouteThreads) s_hist[q] += s_excl[q];     // totals per physical slot
@@ -476,7 +524,7 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
     // epoch (it published before this tile could finish): arm the next step
     if (tid == 0) {
         p.ctl->ticket = 0;
-        unsigned next = (unsigned)epoch + 1u;
+        unsigned next = epoch + 1u;
         p.ctl->epoch = next ? next : 1u;
     }
 }

@@ -17,6 +17,8 @@ struct ScatterParams {
     const uint4 *x;               // [T, H/8] 16-byte units
     uint4 *send;                  // [T*k, H/8]
     int T, k, hv;                 // hv = H/8 (uint4 per row)
+    int P;                        // physical slots
+    unsigned spin_limit;          // polls before a bounded wait gives up
     const int32_t *topk_slot;     // [T,k]
     const int32_t *slot_offsets;  // [P+1]
     const int32_t *pos_in_slot;   // [T*k] stable rank inside the slot (routing kernel's scratch)
@@ -27,19 +29,24 @@ struct ScatterParams {
 
 constexpr int kScatterThreads = 256;
 
-// a9 (final step): row = slot_offsets[slot] + rank inside the slot.  Lane j < k
+// Last step of the permutation: row = slot_offsets[slot] + rank inside the slot.  Lane j < k
 // owns assignment t*k + j.  Only read-only inputs are used, so any number of
 // warps may resolve the same token; exactly one of them writes the result.
+// A slot or row outside its range (possible only if the routing kernel gave up and left
+// stale indices behind) yields -1: the assignment is recorded as not placed and no row is written.
 __device__ __forceinline__ int resolve_row(const ScatterParams &p, int t, int lane, bool write_back)
 {
-    int row = 0;
+    int row = -1;
     if (lane < p.k) {
         const size_t i = (size_t)t * p.k + lane;
         const int slot = __ldg(p.topk_slot + i);
-        row = __ldg(p.slot_offsets + slot) + __ldg(p.pos_in_slot + i);
+        if ((unsigned)slot < (unsigned)p.P) {
+            const long long r = (long long)__ldg(p.slot_offsets + slot) + __ldg(p.pos_in_slot + i);
+            if (r >= 0 && r < (long long)p.T * p.k) row = (int)r;
+        }
         if (write_back) {
             p.dst_row[i] = row;
-            p.src_index[row] = (int)i;
+            if (row >= 0) p.src_index[row] = (int)i;
         }
     }
     return row;
@@ -77,6 +84,7 @@ __global__ void __launch_bounds__(kScatterThreads) k_scatter_vec(ScatterParams p
         const int row = resolve_row(p, t, lane, it % chunks == 0);
         for (int j = 0; j < p.k; ++j) {
             const int r = __shfl_sync(full, row, j);
+            if (r < 0) continue;
             uint4 *dst = p.send + (size_t)r * p.hv;
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u)
@@ -120,6 +128,7 @@ __global__ void __launch_bounds__(kBulkThreads) k_scatter_bulk(ScatterParams p, 
         }
     }
     bool ok = true;
+    int n_failed_at = 0;
     for (int n = 0; n < n_mine && ok; ++n) {
         const int t = first + n * step;
         const int s = n % stages;
@@ -141,16 +150,24 @@ __global__ void __launch_bounds__(kBulkThreads) k_scatter_bulk(ScatterParams p, 
         const unsigned parity = (unsigned)(n / stages) & 1u;
         unsigned spins = 0;
         while (!mbar_try_wait(&full_bar[s], parity)) {
-            if (++spins > kSpinLimit) { ok = false; break; }
+            if (++spins > p.spin_limit) { ok = false; break; }
         }
         ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        if (lane < p.k) {
+        if (!ok) { n_failed_at = n; break; }
+        if (lane < p.k && row >= 0) {
             bulk_store(p.send + (size_t)row * p.hv, ring + (size_t)s * stage_bytes, row_bytes);
             bulk_commit();
         }
     }
-    if (!ok && lane == 0) report_status(p.ctl, kDevTimeout);
+    if (!ok) {
+        if (lane == 0) report_status(p.ctl, kDevTimeout);
+        // loads requested for tokens n_failed_at .. n_failed_at+stages-1 may still be landing in this
+        // CTA's shared memory: give each a bounded chance to finish before the memory is released
+        for (int m = n_failed_at; m < min(n_mine, n_failed_at + stages); ++m) {
+            unsigned spins = 0;
+            while (!mbar_try_wait(&full_bar[m % stages], (unsigned)(m / stages) & 1u) && ++spins < p.spin_limit) {}
+        }
+    }
     bulk_wait_all();   // nothing of this CTA may still read the ring or write HBM at exit
 }
 

@@ -26,10 +26,14 @@ def bf16_bits(t: torch.Tensor) -> np.ndarray:
     return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
 
 
-def make_router(wl, inp, max_tokens, hidden=None, route_scale=1.0) -> B.MoeRouter:
+def make_router(wl, inp, max_tokens, hidden=None, route_scale=1.0, tuning=None) -> B.MoeRouter:
+    """`tuning`: {moe_tuning_option: value} applied right after the context is created."""
     cfg = B.config_for_workload(wl, max_tokens=max_tokens, hidden=hidden, route_scale=route_scale)
     bias = inp["bias"] if wl.score_func == W.SIGMOID else None
-    return B.MoeRouter(cfg, inp["slot_to_expert"], bias, inp["slot_scale"])
+    router = B.MoeRouter(cfg, inp["slot_to_expert"], bias, inp["slot_scale"])
+    for option, value in (tuning or {}).items():
+        router.set_tuning(option, value)
+    return router
 
 
 def assert_y_close(got_bits: np.ndarray, want_bits: np.ndarray):
@@ -50,12 +54,12 @@ def check_dispatch(out: B.DispatchBuffers, ref: dict, check_send=True):
         assert np.array_equal(bf16_bits(out.send_buf), ref["send_buf"]), "send_buf"
 
 
-def run_and_check(wl, inp, failed, router=None, route_scale=1.0):
+def run_and_check(wl, inp, failed, router=None, route_scale=1.0, tuning=None):
     """Dispatch + combine on the GPU, compare everything with the oracle."""
     T, H = inp["x"].shape
     own = router is None
     if own:
-        router = make_router(wl, inp, max_tokens=max(T, 1), hidden=H, route_scale=route_scale)
+        router = make_router(wl, inp, max_tokens=max(T, 1), hidden=H, route_scale=route_scale, tuning=tuning)
         router.set_failed_ranks(failed)
     logits, x = to_dev(inp["logits"]), to_dev(inp["x"], torch.bfloat16)
     out = router.dispatch(logits, x)

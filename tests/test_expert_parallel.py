@@ -275,6 +275,24 @@ def test_receive_buffer_overflow_is_reported_and_nothing_is_written_outside():
     assert all(code == B.MOE_ERR_CAPACITY for code in group.device_status())
     for b in guarded:
         assert bool((b[rows:] == 7.0).all())
+    # The combine that follows (in a captured group step the host cannot step in between) must
+    # not follow the rows that did not fit: they are recorded as dst_row = -1 and contribute
+    # zero, so y is the closed form c_t * x restricted to the rows that were placed.
+    ys = group.combine(T_list)
+    torch.cuda.synchronize()
+    for g, (inp, out, y) in enumerate(zip(inps, group.outs, ys)):
+        dst = out.dst_row.cpu().numpy().reshape(-1, wl.k)
+        assert ((dst >= -1) & (dst < rows)).all() and (dst == -1).any()
+        w = out.topk_weights.cpu().numpy().astype(np.float64)
+        scale = inps[0]["slot_scale"].astype(np.float64)[out.topk_slot.cpu().numpy()]   # the group's scales
+        c = w * scale * (dst >= 0)
+        want = c.sum(1)[:, None] * W.bf16_bits_to_f32(inp["x"]).astype(np.float64)
+        got = y.float().cpu().numpy().astype(np.float64)
+        assert np.isfinite(got).all()
+        err = np.abs(got - want)
+        assert ((err <= 1e-2 * np.abs(want)) | (err <= 1e-3)).all()
+    for b in guarded:
+        assert bool((b[rows:] == 7.0).all())
     group.close()
 
 

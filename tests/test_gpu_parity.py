@@ -37,9 +37,11 @@ def test_parity_full_size(name):
     run_and_check(wl, inp, wl.failure_sets[-1])
 
 
-def test_parity_full_size_kimi_sampled():
-    # 32768 x 7168 with 448 slots: integer outputs compared in full; the 3.7 GB send buffer
-    # and the combine are checked on sampled tokens the oracle computes one by one
+def test_parity_full_size_kimi():
+    # 32768 x 7168 with 448 slots, every output compared in full.  The 3.7 GB send buffer is
+    # compared on the device against the rows the oracle's permutation names (a bit copy of
+    # x[src_index // k]); the combined output y of all 32768 tokens is compared with the oracle,
+    # which computes it chunk by chunk from those same rows.
     wl = W.WORKLOADS["kimi"]
     inp = W.make_inputs(wl)
     failed = wl.failure_sets[3]
@@ -55,18 +57,21 @@ def test_parity_full_size_kimi_sampled():
     ref = oracle.permutation(cfg, slot)
     ref.update(topk_ids=ids, topk_weights=w, topk_slot=slot)
     check_dispatch(out, ref, check_send=False)
-    rng = np.random.default_rng(0)
-    ts = np.unique(np.concatenate([[0, 1, 31, 32, wl.T - 1], rng.integers(0, wl.T, 200)]))
-    rows = ref["dst_row"].reshape(wl.T, wl.k)[ts].reshape(-1)
-    sub = bf16_bits(out.send_buf[torch.from_numpy(rows).cuda().long()])
-    assert np.array_equal(sub, np.repeat(inp["x"][ts], wl.k, axis=0))
-    ref_y = oracle.combine(sub, np.arange(rows.size, dtype=np.int32), w[ts], slot[ts], inp["slot_scale"])
-    assert_y_close(bf16_bits(y[torch.from_numpy(ts).cuda().long()]), ref_y)
-    # whole-buffer property: every row is the bit copy of its source token
-    src_tok = (out.src_index.long() // wl.k)
+    # send buffer: row r is the bit copy of token ref.src_index[r] // k
+    src_tok = torch.from_numpy(ref["src_index"].astype(np.int64) // wl.k).cuda()
     for lo in range(0, wl.T * wl.k, 1 << 16):
         hi = min(lo + (1 << 16), wl.T * wl.k)
         assert torch.equal(out.send_buf[lo:hi].view(torch.int16), x[src_tok[lo:hi]].view(torch.int16))
+    # y: the oracle's combine on every token, 2048 tokens at a time (the rows of a chunk are its
+    # tokens' x rows repeated k times, in assignment order)
+    y_bits = bf16_bits(y)
+    step = 2048
+    for lo in range(0, wl.T, step):
+        hi = min(lo + step, wl.T)
+        rows = np.repeat(inp["x"][lo:hi], wl.k, axis=0)
+        ref_y = oracle.combine(rows, np.arange(rows.shape[0], dtype=np.int32), w[lo:hi], slot[lo:hi],
+                               inp["slot_scale"])
+        assert_y_close(y_bits[lo:hi], ref_y)
     router.close()
 
 
@@ -149,36 +154,50 @@ def test_route_scale():
 
 
 def test_bulk_copy_scatter_matches_oracle():
-    os.environ["MOE_SCATTER_IMPL"] = "1"
-    try:
-        for name, T in (("dsv3", 1037), ("tiny", 128), ("qwen3", 300)):
-            wl = W.WORKLOADS[name]
-            inp = W.make_inputs(wl, T=T)
-            run_and_check(wl, inp, wl.failure_sets[-1])
-        for stages in ("1", "2", "8"):
-            os.environ["MOE_BULK_STAGES"] = stages
-            wl = W.WORKLOADS["dsv3"]
-            run_and_check(wl, W.make_inputs(wl, T=2048 + 5, H=1024), (7,))
-    finally:
-        os.environ.pop("MOE_SCATTER_IMPL", None)
-        os.environ.pop("MOE_BULK_STAGES", None)
+    bulk = {B.MOE_TUNE_SCATTER_IMPL: 1}
+    for name, T in (("dsv3", 1037), ("tiny", 128), ("qwen3", 300)):
+        wl = W.WORKLOADS[name]
+        inp = W.make_inputs(wl, T=T)
+        run_and_check(wl, inp, wl.failure_sets[-1], tuning=bulk)
+    for stages in (1, 2, 8):
+        wl = W.WORKLOADS["dsv3"]
+        run_and_check(wl, W.make_inputs(wl, T=2048 + 5, H=1024), (7,),
+                      tuning={**bulk, B.MOE_TUNE_SCATTER_BULK_STAGES: stages})
 
 
 def test_combine_variants_match_oracle():
     # the register (vector-load) combine and other shapes of the bulk-copy ring
-    settings = [{"MOE_COMBINE_IMPL": "0"},
-                {"MOE_COMBINE_IMPL": "1", "MOE_COMBINE_U": "2", "MOE_COMBINE_STAGES": "2"},
-                {"MOE_COMBINE_IMPL": "1", "MOE_COMBINE_U": "2", "MOE_COMBINE_STAGES": "6"},
-                {"MOE_COMBINE_IMPL": "1", "MOE_COMBINE_U": "4", "MOE_COMBINE_STAGES": "2"}]
-    for env in settings:
-        os.environ.update(env)
-        try:
-            for name, T, H in (("dsv3", 1037, None), ("mixtral", 300, 1000), ("tiny", 128, None), ("qwen3", 5, 8)):
-                wl = W.WORKLOADS[name]
-                run_and_check(wl, W.make_inputs(wl, T=T, H=H), wl.failure_sets[-1])
-        finally:
-            for key in env:
-                os.environ.pop(key, None)
+    settings = [{B.MOE_TUNE_COMBINE_IMPL: 0},
+                {B.MOE_TUNE_COMBINE_IMPL: 1, B.MOE_TUNE_COMBINE_CHUNK: 2, B.MOE_TUNE_COMBINE_STAGES: 2},
+                {B.MOE_TUNE_COMBINE_IMPL: 1, B.MOE_TUNE_COMBINE_CHUNK: 2, B.MOE_TUNE_COMBINE_STAGES: 6},
+                {B.MOE_TUNE_COMBINE_IMPL: 1, B.MOE_TUNE_COMBINE_CHUNK: 4, B.MOE_TUNE_COMBINE_STAGES: 2}]
+    for tuning in settings:
+        for name, T, H in (("dsv3", 1037, None), ("mixtral", 300, 1000), ("tiny", 128, None), ("qwen3", 5, 8)):
+            wl = W.WORKLOADS[name]
+            run_and_check(wl, W.make_inputs(wl, T=T, H=H), wl.failure_sets[-1], tuning=tuning)
+
+
+def test_routing_tile_and_lane_overrides_match_oracle():
+    # other tile sizes (several tiles per SM count, one big tile) and 8 lanes per token
+    wl = W.WORKLOADS["dsv3"]
+    inp = W.make_inputs(wl, T=1037, H=256)
+    for tuning in ({B.MOE_TUNE_ROUTE_TOKENS_PER_TILE: 8}, {B.MOE_TUNE_ROUTE_TOKENS_PER_TILE: 500},
+                   {B.MOE_TUNE_ROUTE_LANES_PER_TOKEN: 8}, {B.MOE_TUNE_PDL: 0}):
+        run_and_check(wl, inp, (7, 20), tuning=tuning)
+
+
+def test_two_contexts_of_different_top_k_share_the_ring_kernel():
+    # both shapes use the generic-k instantiation of the ring combine with different ring sizes;
+    # creating the second context must not shrink what the first may launch with
+    wl16 = W.Workload("k16", T=64, H=512, E=64, k=16, R=8, S=8, seed=5, max_replicas=1)
+    wl6 = W.Workload("k6", T=64, H=512, E=64, k=6, R=8, S=8, seed=6, max_replicas=1)
+    inp16, inp6 = W.make_inputs(wl16), W.make_inputs(wl6)
+    r16 = make_router(wl16, inp16, max_tokens=64)
+    r6 = make_router(wl6, inp6, max_tokens=64)
+    for _ in range(2):
+        run_and_check(wl16, inp16, (), router=r16)
+        run_and_check(wl6, inp6, (), router=r6)
+    r16.close(); r6.close()
 
 
 def test_step_from_host_memory():

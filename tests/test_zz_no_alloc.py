@@ -1,4 +1,4 @@
-"""The allocation-free entry point (`moe_permute_static`) against the regular path.
+"""The allocation-free entry point (`moe_permute_static`) against the regular path and the oracle.
 
 Some users of the library run inside a process that may not allocate device
 memory after start-up (for instance a serving engine that has already claimed
@@ -6,8 +6,10 @@ all of HBM for its own pool).  They cannot build a context, so they call
 `moe_permute_static`, which keeps its scratch in a fixed array inside the
 library.  Here its counts, offsets and permutation are compared, bit for bit
 (they are integers), with what `moe_dispatch` produces for the same slot
-assignments — twice in a row with different inputs, because the second call
-finds the first call's leftovers in the shared scratch.
+assignments AND with the CPU oracle's permutation of those assignments — twice
+in a row with different inputs, because the second call finds the first call's
+leftovers in the shared scratch.  The second call is also watched for device
+allocations: the free-memory figure of the device must not move across it.
 
 This file is named so that pytest collects it last.
 """
@@ -15,9 +17,11 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2602_21140_b200 import binding as B
 from paper_2602_21140_b200 import workloads as W
 from gpu_util import make_router, to_dev
+from util import oracle_cfg
 
 pytestmark = pytest.mark.gpu
 
@@ -48,16 +52,34 @@ def _regular_dispatch(wl, T, failed, seed):
     return out
 
 
-def test_two_calls_in_a_row_match_the_regular_path():
+def test_two_calls_in_a_row_match_the_regular_path_and_the_oracle():
     # first call: large, skewed, 448 slots; second call: smaller and a different layout, so
     # stale histogram rows of the first call sit in the scratch the second call uses
-    for name, T, failed, seed in (("kimi", 5000 + 13, (3, 40), 21), ("dsv3", 1037, (7, 20), 22)):
+    for call, (name, T, failed, seed) in enumerate((("kimi", 5000 + 13, (3, 40), 21), ("dsv3", 1037, (7, 20), 22))):
         wl = W.WORKLOADS[name]
         out = _regular_dispatch(wl, T, failed, seed)
-        got = _static_permute(wl, out.topk_slot.reshape(-1))
+        slots = out.topk_slot.reshape(-1)
+        if call == 0:
+            got = _static_permute(wl, slots)
+        else:
+            # by now the library's device code is loaded and the scratch address is known: this
+            # call must leave the device's free memory exactly where it was (torch's own output
+            # tensors are created before the first reading and stay alive past the second)
+            warm = _static_permute(wl, slots)
+            torch.cuda.synchronize()
+            free_before = torch.cuda.mem_get_info()[0]
+            st = B.moe_permute_static(slots.data_ptr(), slots.numel(), wl.R, wl.S,
+                                      *(warm[f].data_ptr() for f in FIELDS),
+                                      torch.cuda.current_stream().cuda_stream)
+            torch.cuda.synchronize()
+            assert st == B.MOE_OK
+            assert torch.cuda.mem_get_info()[0] == free_before, "moe_permute_static allocated device memory"
+            got = warm
         torch.cuda.synchronize()
+        ref = oracle.permutation(oracle_cfg(wl), slots.cpu().numpy().reshape(T, wl.k))
         for f in FIELDS:
             assert torch.equal(got[f], getattr(out, f).reshape(-1)), (name, f)
+            assert np.array_equal(got[f].cpu().numpy(), ref[f].reshape(-1)), (name, f, "oracle")
 
 
 def test_sizes_beyond_the_built_in_scratch_are_refused():
