@@ -19,9 +19,9 @@ constexpr unsigned kDefaultSpinLimit = 1u << 20;
 constexpr unsigned kSpinSleepNs = 64;
 
 struct Control {
-    unsigned ticket;   // next tile of the running routing kernel
-    unsigned epoch;    // step counter tagging the look-back descriptors
-    int status;        // kDev* code, sticky until the host clears it
+    unsigned ticket;     // next tile of the running routing kernel
+    unsigned epoch;      // step counter tagging the per-tile count rows
+    int status;          // kDev* code, sticky until the host clears it
     int pad;
 };
 
@@ -43,35 +43,19 @@ __device__ __forceinline__ unsigned lanemask_lt()
     return m;
 }
 
-__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long *p)
+// A pair of 64-bit words moved by one 16-byte access at GPU scope.  Each word is read and
+// written whole (a reader never sees half of one), which is all the look-back needs: every
+// word carries its own validity tag.
+__device__ __forceinline__ ulonglong2 ld_relaxed_v2_u64(const ulonglong2 *p)
 {
-    unsigned long long v;
-    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    ulonglong2 v;
+    asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(v.x), "=l"(v.y) : "l"(p) : "memory");
     return v;
 }
 
-__device__ __forceinline__ void st_relaxed_u64(unsigned long long *p, unsigned long long v)
+__device__ __forceinline__ void st_relaxed_v2_u64(ulonglong2 *p, unsigned long long a, unsigned long long b)
 {
-    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
-}
-
-__device__ __forceinline__ unsigned ld_relaxed_u32(const unsigned *p)
-{
-    unsigned v;
-    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
-
-__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p)
-{
-    unsigned v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
-
-__device__ __forceinline__ void st_relaxed_u32(unsigned *p, unsigned v)
-{
-    asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+    asm volatile("st.relaxed.gpu.global.v2.u64 [%0], {%1, %2};" ::"l"(p), "l"(a), "l"(b) : "memory");
 }
 
 __device__ __forceinline__ int ld_relaxed_s32(const int *p)

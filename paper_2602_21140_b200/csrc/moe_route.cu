@@ -216,9 +216,8 @@ struct moe_ctx {
     int32_t *d_live;           // live-replica lists derived from d_state (k_derive_live)
     float *d_bias;
     float *d_slot_scale;
-    uint16_t *d_tile_counts;   // [tiles][p_pad] per-tile, per-slot counts of the running step
-    unsigned *d_tile_flag;     // [tiles] epoch of the step that published the row
-    size_t scan_tiles;         // rows the two arrays above were allocated for
+    ulonglong2 *d_tile_counts; // [tiles][p_pad/4] epoch-tagged per-tile, per-slot counts of the running step
+    size_t scan_tiles;         // rows the array above was allocated for
     moe::Control *d_ctl;
     int32_t *d_pos;
     uint4 *d_zero_row;         // [H/8] zeros: source of an assignment that was not placed
@@ -262,7 +261,7 @@ size_t device_bytes_for(const Derived &d, int max_tokens)
     b += (size_t)d.state_words * 4;
     b += (size_t)d.E * (1 + d.max_rep) * 4;
     b += (size_t)d.E * 4 + (size_t)d.P * 4;
-    b += tiles * d.p_pad * sizeof(uint16_t) + tiles * sizeof(unsigned);
+    b += tiles * (d.p_pad / 4) * sizeof(ulonglong2);
     b += sizeof(moe::Control);
     b += (size_t)max_tokens * d.k * 4;
     b += (size_t)d.H * 2;
@@ -357,7 +356,7 @@ cudaError_t enqueue_route(moe_ctx *ctx, const float *logits, int32_t T, const mo
     rp.pos_in_slot = ctx->d_pos;
     rp.slot_counts = out->slot_counts; rp.slot_offsets = out->slot_offsets;
     rp.rank_counts = out->rank_counts; rp.rank_offsets = out->rank_offsets;
-    rp.tile_counts = ctx->d_tile_counts; rp.tile_flag = ctx->d_tile_flag; rp.ctl = ctx->d_ctl;
+    rp.tile_counts = ctx->d_tile_counts; rp.ctl = ctx->d_ctl;
     const int tiles = (T + d.tokens_per_block - 1) / d.tokens_per_block;
     return launch_route(d.epl, d.lpt, rp, tiles, ctx->route_smem, st, ctx->pdl);
 }
@@ -428,21 +427,20 @@ bool stream_is_capturing(cudaStream_t st)
     return cs != cudaStreamCaptureStatusNone;
 }
 
-// (Re)allocate the per-tile count rows and flags for the context's current tile size.
+// (Re)allocate the per-tile count rows for the context's current tile size.
 bool alloc_scan_scratch(moe_ctx *ctx, cudaStream_t st)
 {
     const Derived &d = ctx->d;
     const size_t tiles = ((size_t)ctx->cfg.max_tokens + d.tokens_per_block - 1) / d.tokens_per_block;
+    const size_t row = (size_t)(d.p_pad / 4) * sizeof(ulonglong2);
     if (tiles > ctx->scan_tiles) {
-        cudaFree(ctx->d_tile_counts); cudaFree(ctx->d_tile_flag);
-        ctx->d_tile_counts = nullptr; ctx->d_tile_flag = nullptr; ctx->scan_tiles = 0;
-        if (cudaMalloc(&ctx->d_tile_counts, tiles * d.p_pad * sizeof(uint16_t)) != cudaSuccess ||
-            cudaMalloc(&ctx->d_tile_flag, tiles * sizeof(unsigned)) != cudaSuccess)
-            return false;
+        cudaFree(ctx->d_tile_counts);
+        ctx->d_tile_counts = nullptr; ctx->scan_tiles = 0;
+        if (cudaMalloc(&ctx->d_tile_counts, tiles * row) != cudaSuccess) return false;
         ctx->scan_tiles = tiles;
     }
-    // flag 0 never equals an epoch (epochs start at 1 and skip 0)
-    return cudaMemsetAsync(ctx->d_tile_flag, 0, ctx->scan_tiles * sizeof(unsigned), st) == cudaSuccess;
+    // tag 0 never equals an epoch (epochs start at 1 and skip 0)
+    return cudaMemsetAsync(ctx->d_tile_counts, 0, ctx->scan_tiles * row, st) == cudaSuccess;
 }
 
 // The kernels with rings in dynamic shared memory may use all of it.  The attribute belongs to
@@ -528,7 +526,7 @@ void free_ctx(moe_ctx *ctx)
 {
     if (!ctx) return;
     cudaFree(ctx->d_state); cudaFree(ctx->d_live); cudaFree(ctx->d_bias); cudaFree(ctx->d_slot_scale);
-    cudaFree(ctx->d_tile_counts); cudaFree(ctx->d_tile_flag); cudaFree(ctx->d_ctl); cudaFree(ctx->d_pos);
+    cudaFree(ctx->d_tile_counts); cudaFree(ctx->d_ctl); cudaFree(ctx->d_pos);
     cudaFree(ctx->d_zero_row);
     cudaFree(ctx->d_peer_bufs); cudaFree(ctx->d_src_base);
     for (int s = 0; s < kStagingSlots; ++s) {
@@ -622,7 +620,7 @@ moe_status moe_route_init(const moe_config *cfg, const int32_t *slot_to_expert, 
         ctx->h_stage[s] = nullptr; ctx->stage_done[s] = nullptr; ctx->stage_used[s] = false;
     }
     ctx->d_state = nullptr; ctx->d_live = nullptr; ctx->d_bias = nullptr; ctx->d_slot_scale = nullptr;
-    ctx->d_tile_counts = nullptr; ctx->d_tile_flag = nullptr; ctx->scan_tiles = 0;
+    ctx->d_tile_counts = nullptr; ctx->scan_tiles = 0;
     ctx->d_ctl = nullptr; ctx->d_pos = nullptr; ctx->d_zero_row = nullptr;
     for (int i = 0; i < kNumTuning; ++i) ctx->tune[i] = -1;
 

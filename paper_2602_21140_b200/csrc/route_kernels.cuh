@@ -14,10 +14,11 @@
 // Prefix over tiles: the whole problem fits in one wave of CTAs (the host sizes the
 // tile so that a step has about one tile per SM), so all tiles publish at about the
 // same time and a chained look-back (wait for the predecessor's inclusive prefix)
-// would serialise them.  Instead every tile publishes only its own per-slot counts
-// (16-bit, eight to a 16-byte store) followed by one flag word carrying the step's
-// epoch, waits for the flags of ALL earlier tiles (one polling thread per tile) and
-// sums their counts with independent 16-byte loads: two L2 round trips in all.
+// would serialise them.  Instead every tile publishes only its own per-slot counts,
+// two 16-bit counts and the step's 32-bit epoch to a 64-bit word (the epoch makes a stale
+// word invalid without any clearing, and data and validity arrive in one load), and sums
+// the counts of ALL earlier tiles with independent 16-byte loads: one L2 round trip when
+// the other tiles have already published.
 #pragma once
 
 #include "device_utils.cuh"
@@ -36,8 +37,8 @@ constexpr int kRouteWarps = kRouteThreads / 32;
 //                        layout (logical-rank order; identity unless ranks were compacted)
 constexpr int kStateHeaderWords = 2;
 
-// A step has at most this many tiles (one polling thread per earlier tile in the look-back).
-constexpr int kMaxRouteTiles = kRouteThreads;
+// A step has at most this many tiles.
+constexpr int kMaxRouteTiles = 1024;
 
 // Live-replica lists derived from the state blob: per expert 1 + max_rep words, the number of
 // live replicas followed by their slots in ascending order.  k_derive_live rebuilds them on
@@ -88,8 +89,8 @@ struct RouteParams {
     int32_t *topk_slot;       // [T,k]
     int32_t *pos_in_slot;     // [T*k]: stable rank of assignment i inside its slot
     int32_t *slot_counts, *slot_offsets, *rank_counts, *rank_offsets;
-    uint16_t *tile_counts;    // [tiles][p_pad]: assignments of each tile on each slot
-    unsigned *tile_flag;      // [tiles]: epoch of the step whose counts the row holds
+    ulonglong2 *tile_counts;  // [tiles][p_pad/4]: per tile, four slots to a 16-byte entry: two words
+                              // of (epoch << 32 | count of the odd slot << 16 | count of the even slot)
     Control *ctl;
 };
 
@@ -408,73 +409,78 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
     }
 
     // ---- prefix over tiles: publish this tile's counts, sum those of all earlier tiles
+    const int groups = p.p_pad / 4;                        // 16-byte entries per tile row
     {
-        uint4 *mine = reinterpret_cast<uint4 *>(p.tile_counts + (size_t)ticket * p.p_pad);
-        for (int q8 = tid; q8 < p.p_pad / 8; q8 += kRouteThreads) {
-            const int32_t *h = s_hist + 8 * q8;            // entries past P stay zero
-            uint4 v;
-            v.x = (unsigned)h[0] | ((unsigned)h[1] << 16); v.y = (unsigned)h[2] | ((unsigned)h[3] << 16);
-            v.z = (unsigned)h[4] | ((unsigned)h[5] << 16); v.w = (unsigned)h[6] | ((unsigned)h[7] << 16);
-            __stcg(mine + q8, v);
+        ulonglong2 *mine = p.tile_counts + (size_t)ticket * groups;
+        const unsigned long long tag = (unsigned long long)epoch << 32;
+        for (int q4 = tid; q4 < groups; q4 += kRouteThreads) {
+            const int32_t *h = s_hist + 4 * q4;            // entries past P stay zero
+            st_relaxed_v2_u64(mine + q4, tag | (unsigned)h[0] | ((unsigned)h[1] << 16),
+                              tag | (unsigned)h[2] | ((unsigned)h[3] << 16));
         }
-    }
-    __syncthreads();
-    if (tid == 0) {
-        __threadfence();                                   // the counts of every thread, then the flag
-        st_relaxed_u32(p.tile_flag + ticket, epoch);
     }
     if (ticket > 0) {
-        // one thread per earlier tile waits for that tile's flag
+        // thread = (segment g of the earlier tiles, entry q4); every load is independent of the others
+        const int nseg = kRouteThreads / groups;           // >= 1: P <= 4096
+        const int g = tid / groups, q4 = tid % groups;
         bool gave_up = false;
-        if (tid < (int)ticket) {
-            unsigned spins = 0;
-            while (ld_acquire_u32(p.tile_flag + tid) != epoch) {
-                if (++spins > p.spin_limit ||
-                    ((spins & 255u) == 0 && ld_relaxed_s32(&p.ctl->status) == kDevTimeout)) {
-                    gave_up = true;
-                    break;
+        int acc[4] = {0, 0, 0, 0};
+        if (g < nseg) {
+            // Up to kBatch entries are requested together and the stale ones (their tile has not
+            // published yet) are requested again together, so a round of retries costs one trip
+            // to L2 however many of the entries were stale.
+            constexpr int kBatch = 6;
+            for (int b0 = g; b0 < (int)ticket && !gave_up; b0 += nseg * kBatch) {
+                ulonglong2 v[kBatch];
+                unsigned pending = 0;
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u)
+                    if (b0 + u * nseg < (int)ticket) pending |= 1u << u;
+                unsigned spins = 0;
+                while (true) {
+#pragma unroll
+                    for (int u = 0; u < kBatch; ++u)
+                        if ((pending >> u) & 1u)
+                            v[u] = ld_relaxed_v2_u64(p.tile_counts + (size_t)(b0 + u * nseg) * groups + q4);
+#pragma unroll
+                    for (int u = 0; u < kBatch; ++u) {
+                        if (((pending >> u) & 1u) && (unsigned)(v[u].x >> 32) == epoch &&
+                            (unsigned)(v[u].y >> 32) == epoch) {
+                            acc[0] += (int)(v[u].x & 0xffffu); acc[1] += (int)((v[u].x >> 16) & 0xffffu);
+                            acc[2] += (int)(v[u].y & 0xffffu); acc[3] += (int)((v[u].y >> 16) & 0xffffu);
+                            pending &= ~(1u << u);
+                        }
+                    }
+                    if (pending == 0) break;
+                    if (++spins > p.spin_limit ||
+                        ((spins & 255u) == 0 && ld_relaxed_s32(&p.ctl->status) == kDevTimeout)) {
+                        gave_up = true;
+                        break;
+                    }
+                    if (spins > 4) __nanosleep(kSpinSleepNs);
                 }
-                __nanosleep(kSpinSleepNs);
             }
         }
+        if (groups <= 16 && (groups & (groups - 1)) == 0) {
+            // few slots: lanes q4, q4 + groups, ... of a warp hold partial sums of the same
+            // entry; add them up in registers before touching shared memory
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                for (int off = groups; off < 32; off <<= 1) acc[u] += __shfl_xor_sync(full, acc[u], off);
+            if (lane >= groups) { acc[0] = acc[1] = acc[2] = acc[3] = 0; }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (acc[u]) atomicAdd(&s_excl[4 * q4 + u], acc[u]);
         if (__syncthreads_or(gave_up)) {
             // An earlier tile never published.  Nothing of this tile's placement is written, the
             // control word stays as it is, and the status word tells the host (which re-arms it).
             if (tid == 0) report_status(p.ctl, kDevTimeout);
             return;
         }
-        // thread = (segment g of the earlier tiles, group q8 of eight slots); every load is independent
-        const int groups = p.p_pad / 8;
-        const int nseg = kRouteThreads / groups;           // >= 2: P <= 4096
-        const int g = tid / groups, q8 = tid % groups;
-        if (g < nseg) {
-            constexpr int kBatch = 4;
-            int acc[8];
-#pragma unroll
-            for (int u = 0; u < 8; ++u) acc[u] = 0;
-            for (int b0 = g; b0 < (int)ticket; b0 += nseg * kBatch) {
-                uint4 v[kBatch];
-#pragma unroll
-                for (int u = 0; u < kBatch; ++u) {
-                    const int b = b0 + u * nseg;
-                    v[u] = make_uint4(0u, 0u, 0u, 0u);
-                    if (b < (int)ticket)
-                        v[u] = __ldcg(reinterpret_cast<const uint4 *>(p.tile_counts + (size_t)b * p.p_pad) + q8);
-                }
-#pragma unroll
-                for (int u = 0; u < kBatch; ++u) {
-                    acc[0] += v[u].x & 0xffffu; acc[1] += v[u].x >> 16;
-                    acc[2] += v[u].y & 0xffffu; acc[3] += v[u].y >> 16;
-                    acc[4] += v[u].z & 0xffffu; acc[5] += v[u].z >> 16;
-                    acc[6] += v[u].w & 0xffffu; acc[7] += v[u].w >> 16;
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < 8; ++u)
-                if (acc[u]) atomicAdd(&s_excl[8 * q8 + u], acc[u]);
-        }
+    } else {
+        __syncthreads();
     }
-    __syncthreads();
 
     // stable rank of every assignment of the tile inside its slot, over all tiles
     for (int i = tid; i < n_tok * k; i += kRouteThreads)
