@@ -65,6 +65,22 @@ __device__ __forceinline__ int ld_relaxed_s32(const int *p)
     return v;
 }
 
+// Asynchronous copies global -> shared that bypass registers; wait_all covers the calling
+// thread's own copies (enough when the same thread reads what it asked for).
+__device__ __forceinline__ void cp_async_16(void *smem_dst, const void *gsrc)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc)
+                 : "memory");
+}
+
+__device__ __forceinline__ void cp_async_4(void *smem_dst, const void *gsrc)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc)
+                 : "memory");
+}
+
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
 __device__ __forceinline__ void report_status(Control *ctl, int code)
 {
     atomicCAS(&ctl->status, kDevOk, code);   // the first error wins and sticks

@@ -113,9 +113,9 @@ bool derive(const moe_config *c, Derived *d, int want_lpt = 0, int want_tile = 0
     int tile = want_tile > 0 ? want_tile : std::max(32, (c->max_tokens + kRouteTileTarget - 1) / kRouteTileTarget);
     tile = (tile + per_warp - 1) / per_warp * per_warp;
     while (tile > per_warp &&
-           (route_smem_bytes(d->E, d->max_rep, tile, d->k, d->P) > kMaxSmem - 1024 || (long long)tile * d->k > 65535))
+           (route_smem_bytes(d->E, d->max_rep, tile, d->k, d->P, d->epl) > kMaxSmem - 1024 || (long long)tile * d->k > 65535))
         tile = (tile / 2 + per_warp - 1) / per_warp * per_warp;
-    if (route_smem_bytes(d->E, d->max_rep, tile, d->k, d->P) > kMaxSmem - 1024 || (long long)tile * d->k > 65535)
+    if (route_smem_bytes(d->E, d->max_rep, tile, d->k, d->P, d->epl) > kMaxSmem - 1024 || (long long)tile * d->k > 65535)
         return false;
     d->tokens_per_block = tile;
     if ((c->max_tokens + tile - 1) / tile > kMaxRouteTiles) return false;
@@ -476,7 +476,7 @@ int tuned(const moe_ctx *ctx, int option, int dflt)
 void configure_launch(moe_ctx *ctx)
 {
     const Derived &d = ctx->d;
-    ctx->route_smem = route_smem_bytes(d.E, d.max_rep, d.tokens_per_block, d.k, d.P);
+    ctx->route_smem = route_smem_bytes(d.E, d.max_rep, d.tokens_per_block, d.k, d.P, d.epl);
     ctx->spin_limit = (unsigned)tuned(ctx, MOE_TUNE_SPIN_LIMIT, (int)kDefaultSpinLimit);
     ctx->pdl = tuned(ctx, MOE_TUNE_PDL, 1) != 0;
     ctx->scatter_impl = tuned(ctx, MOE_TUNE_SCATTER_IMPL, 0);

@@ -95,40 +95,34 @@ struct RouteParams {
 };
 
 __host__ __device__ inline size_t route_smem_bytes(int E, int max_rep, int tokens_per_block, int k,
-                                                   int P)
+                                                   int P, int epl)
 {
     const size_t p_pad = ((size_t)P + 7) & ~(size_t)7;
-    size_t words = (size_t)E * (1 + max_rep) + 2 * (size_t)tokens_per_block * k + 2 * p_pad + (size_t)P;
+    // per warp: [blocks][32] 16-byte entries (logits, then key codes) and [blocks][32] block bests
+    const size_t code_words = (size_t)kRouteWarps * ((epl + 3) / 4) * 32 * 5;
+    const size_t bias_words = (size_t)((epl + 3) / 4 * 4) * 16 + 16;   // bias by (expert of the lane, lane); availability bits
+    size_t words = code_words + bias_words + (size_t)E * (1 + max_rep) + 2 * (size_t)tokens_per_block * k +
+                   2 * p_pad + (size_t)P;
     return words * sizeof(int32_t) + (size_t)kRouteWarps * P * sizeof(uint16_t);
-}
-
-// Block B (experts 4B..4B+3 of a lane) lost element `taken`: blank it and find the block's
-// next best code, lowest index first among equals.
-template <int B, int EPL>
-__device__ __forceinline__ void rescan_block(uint32_t (&code)[EPL], uint32_t (&bm)[(EPL + 3) / 4],
-                                             int (&bq)[(EPL + 3) / 4], int taken)
-{
-    if constexpr (4 * B < EPL) {
-        uint32_t best = 0; int at = 4 * B;
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            constexpr int q0 = 4 * B;
-            if (q0 + u < EPL) {
-                const uint32_t c = (q0 + u == taken) ? 0u : code[q0 + u];
-                code[q0 + u] = c;
-                if (c > best) { best = c; at = q0 + u; }
-            }
-        }
-        bm[B] = best; bq[B] = at;
-    }
 }
 
 // Route 32/LPT tokens with one warp.  Lanes [sub*LPT, (sub+1)*LPT) own token
 // t_first + sub.  On return, sub-lane j < k of a token holds its j-th chosen
 // expert, the weight and the physical slot.
+//
+// The element work is written as a short loop over blocks of four experts rather than
+// unrolled over all EPL of them: every warp passes through this code about once per
+// launch, and straight-line code that is run once is paced by instruction fetch (the
+// unrolled form measured ~350 cycles per expert with nothing but integer work in it),
+// while a loop body that stays in the instruction cache issues at full rate.  For the loop
+// to be possible nothing may be indexed by the block number in registers, so a lane keeps
+// its logits, then its key codes, and its per-block best codes in its own column of two
+// small shared-memory tables (s_blk[b * 32 + lane], s_bmx[b * 32 + lane]: no two lanes
+// ever touch the same word, so no synchronisation is needed).
 template <int EPL, int LPT>
 __device__ __forceinline__ void route_tokens(const RouteParams &p, int t_first, uint32_t avail_mask,
-                                             const int32_t *s_live, int fallback_expert, int &out_id,
+                                             const int32_t *s_live, const float *s_bias, uint4 *s_blk,
+                                             uint32_t *s_bmx, int fallback_expert, int &out_id,
                                              float &out_w, int &out_slot)
 {
     const unsigned full = 0xffffffffu;
@@ -141,42 +135,58 @@ __device__ __forceinline__ void route_tokens(const RouteParams &p, int t_first, 
     const float neg_inf = __int_as_float(0xff800000);
     const bool sigmoid = p.score_func != 0;
     const bool grouped = p.n_group > 1;
+    constexpr int kBlocks = (EPL + 3) / 4;
+    uint4 *mine = s_blk + lane;
+    uint32_t *mine_bmx = s_bmx + lane;
 
-    // gate scores, availability mask, and the two best keys of this lane (for the group scores)
-    uint32_t code[EPL];
-    float h1 = neg_inf, h2 = neg_inf;
+    // 1. this lane's logits, global -> shared without passing through registers (all requests
+    //    are in flight together; entries past the lane's experts or past E read -inf)
+    if ((EPL % 4 == 0) && (E == LPT * EPL)) {
 #pragma unroll
-    for (int q0 = 0; q0 < EPL; q0 += 4) {
-        float lg[4];
-        if ((EPL % 4 == 0) && (E == LPT * EPL)) {
-            const float4 v = __ldg(reinterpret_cast<const float4 *>(row + e0 + q0));
-            lg[0] = v.x; lg[1] = v.y; lg[2] = v.z; lg[3] = v.w;
-        } else {
+        for (int b = 0; b < kBlocks; ++b) cp_async_16(mine + b * 32, row + e0 + 4 * b);
+    } else {
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
-                lg[u] = (q0 + u < EPL && e0 + q0 + u < E) ? __ldg(row + e0 + q0 + u) : neg_inf;
+        for (int q = 0; q < 4 * kBlocks; ++q) {
+            float *dst = reinterpret_cast<float *>(mine + (q / 4) * 32) + (q % 4);
+            if (q < EPL && e0 + q < E) cp_async_4(dst, row + e0 + q);
+            else *dst = neg_inf;
         }
+    }
+    cp_async_wait_all();
+
+    // 2. gate scores, availability mask, order-preserving key codes (written over the logits),
+    //    the best code of every block, and the two best keys of this lane (for the group scores).
+    //    Four experts per trip: four independent chains of arithmetic keep the pipeline busy,
+    //    and the body still fits the instruction cache.
+    float h1 = neg_inf, h2 = neg_inf;
+    uint32_t lbest = 0; int lb = 0;
+#pragma unroll 1
+    for (int b = 0; b < kBlocks; ++b) {
+        const float4 v = *reinterpret_cast<const float4 *>(mine + b * 32);
+        const float lg[4] = {v.x, v.y, v.z, v.w};
+        uint32_t c[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const int q = q0 + u;
-            if (q < EPL) {
-                float kf = lg[u];
-                if (sigmoid)
-                    kf = __fadd_rn(sigmoid_spec(lg[u]), (e0 + q < E) ? __ldg(p.bias + e0 + q) : 0.0f);
-                const bool ok = ((avail_mask >> q) & 1u) && (lg[u] != neg_inf);
-                kf = ok ? kf : neg_inf;
-                if (grouped) {                            // running two best keys of the lane
-                    h2 = fmaxf(h2, fminf(h1, kf));
-                    h1 = fmaxf(h1, kf);
-                }
-                code[q] = key_code(kf);
+            const int q = 4 * b + u;
+            float kf = lg[u];
+            if (sigmoid) kf = __fadd_rn(sigmoid_spec(lg[u]), s_bias[q * LPT + sl]);
+            const bool ok = ((avail_mask >> q) & 1u) && (lg[u] != neg_inf);
+            kf = ok ? kf : neg_inf;
+            if (grouped) {                                // running two best keys of the lane
+                h2 = fmaxf(h2, fminf(h1, kf));
+                h1 = fmaxf(h1, kf);
             }
+            c[u] = key_code(kf);
         }
+        *(mine + b * 32) = make_uint4(c[0], c[1], c[2], c[3]);
+        const uint32_t bmax = max(max(c[0], c[1]), max(c[2], c[3]));
+        mine_bmx[b * 32] = bmax;
+        if (bmax > lbest) { lbest = bmax; lb = b; }      // lowest block among equals
     }
 
     // group-limited selection: score = sum of the (up to) group_m best finite keys
-    bool active = true;
-    if (p.n_group > 1) {
+    if (grouped) {
+#pragma unroll 1
         for (int off = 1; off < p.lanes_per_group; off <<= 1) {
             const float o1 = __shfl_xor_sync(full, h1, off, LPT);
             const float o2 = __shfl_xor_sync(full, h2, off, LPT);
@@ -187,57 +197,44 @@ __device__ __forceinline__ void route_tokens(const RouteParams &p, int t_first, 
         const float gscore = (p.group_m == 1 || h2 == neg_inf) ? h1 : __fadd_rn(h1, h2);
         const int g = sl / p.lanes_per_group;
         int rank = 0;
+#pragma unroll 1
         for (int gp = 0; gp < p.n_group; ++gp) {
             const float o = __shfl_sync(full, gscore, gp * p.lanes_per_group, LPT);
             rank += (o > gscore) || (o == gscore && gp < g);
         }
-        active = (g < p.n_group) && (rank < p.topk_group);
+        if (!((g < p.n_group) && (rank < p.topk_group))) lbest = 0;   // this lane's group is not kept
     }
 
-    // top-k: k rounds of arg-max over order-preserving integer codes.  A lane keeps the best
-    // code of each block of four of its experts, so that after a pick only the block that lost
-    // an element is scanned again (the rounds are bound by instruction issue).
-    constexpr int kBlocks = (EPL + 3) / 4;
-    uint32_t bm[kBlocks]; int bq[kBlocks];
-#pragma unroll
-    for (int b = 0; b < kBlocks; ++b) {
-        bm[b] = 0; bq[b] = 4 * b;
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int q = 4 * b + u;
-            if (q < EPL && active && code[q] > bm[b]) { bm[b] = code[q]; bq[b] = q; }
-        }
-    }
-    uint32_t lbest = 0; int lq = 0;
-#pragma unroll
-    for (int b = 0; b < kBlocks; ++b)
-        if (bm[b] > lbest) { lbest = bm[b]; lq = bq[b]; }
+    // top-k: k rounds of arg-max over the codes.  A lane offers the best code it has left; the
+    // winner (lowest lane among equals = lowest expert id) reads the block of four that held
+    // it, blanks the first element equal to it (lowest id among equals), and finds its next best
+    // from the per-block bests.
     const unsigned seg_mask = ((LPT == 32) ? 0xffffffffu : ((1u << LPT) - 1u)) << (sub * LPT);
     int my_id = fallback_expert; bool my_bad = false;
+#pragma unroll 1
     for (int j = 0; j < p.k; ++j) {
         const uint32_t m = __reduce_max_sync(seg_mask, lbest);
         const unsigned ball = __ballot_sync(full, lbest == m);
         const int src = __ffs(ball & seg_mask) - 1 - sub * LPT;   // lowest lane = lowest expert id
-        const int sel_e = __shfl_sync(full, e0 + lq, src, LPT);
         const bool bad = m <= kCodeNegInf;               // nothing selectable is left
-        if (sl == j) { my_id = bad ? fallback_expert : sel_e; my_bad = bad; }
+        int taken_e = 0;
         if (sl == src && !bad) {                         // drop the pick, find the lane's next best
-            const int taken = lq;
-            switch (taken >> 2) {
-                case 0: rescan_block<0, EPL>(code, bm, bq, taken); break;
-                case 1: rescan_block<1, EPL>(code, bm, bq, taken); break;
-                case 2: rescan_block<2, EPL>(code, bm, bq, taken); break;
-                case 3: rescan_block<3, EPL>(code, bm, bq, taken); break;
-                case 4: rescan_block<4, EPL>(code, bm, bq, taken); break;
-                case 5: rescan_block<5, EPL>(code, bm, bq, taken); break;
-                case 6: rescan_block<6, EPL>(code, bm, bq, taken); break;
-                default: rescan_block<7, EPL>(code, bm, bq, taken); break;
-            }
-            lbest = 0; lq = 0;
+            const uint4 blk = *(mine + lb * 32);
+            const int u = (blk.x == lbest) ? 0 : (blk.y == lbest) ? 1 : (blk.z == lbest) ? 2 : 3;
+            reinterpret_cast<uint32_t *>(mine + lb * 32)[u] = 0u;
+            taken_e = e0 + lb * 4 + u;
+            const uint32_t c0 = (u == 0) ? 0u : blk.x, c1 = (u == 1) ? 0u : blk.y;
+            const uint32_t c2 = (u == 2) ? 0u : blk.z, c3 = (u == 3) ? 0u : blk.w;
+            mine_bmx[lb * 32] = max(max(c0, c1), max(c2, c3));
+            lbest = 0; lb = 0;
 #pragma unroll
-            for (int b = 0; b < kBlocks; ++b)
-                if (bm[b] > lbest) { lbest = bm[b]; lq = bq[b]; }
+            for (int b = 0; b < kBlocks; ++b) {
+                const uint32_t bm = mine_bmx[b * 32];
+                if (bm > lbest) { lbest = bm; lb = b; }
+            }
         }
+        const int sel_e = __shfl_sync(full, taken_e, src, LPT);
+        if (sl == j) { my_id = bad ? fallback_expert : sel_e; my_bad = bad; }
     }
 
     // weights: ratio of the chosen scores, summed and divided in double.  The score of a
@@ -255,6 +252,7 @@ __device__ __forceinline__ void route_tokens(const RouteParams &p, int t_first, 
         else u = (double)my_val;
     }
     double usum = 0.0;
+#pragma unroll 1
     for (int j = 0; j < p.k; ++j) usum += __shfl_sync(full, u, j, LPT);
     out_w = (float)((double)p.route_scale * u / usum);
 
@@ -275,7 +273,16 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
     const int E = p.E, P = p.P, k = p.k, tb = p.tokens_per_block;
     const int NA = tb * k;
     const int live_words = 1 + p.max_rep;
-    int32_t *s_live = smem;                           // [E][1 + max_rep] live count, live slots
+    constexpr int kBlockEntries = (EPL + 3) / 4 * 32;   // one warp's [blocks][32] table
+    uint4 *s_blk = reinterpret_cast<uint4 *>(smem) + (threadIdx.x >> 5) * kBlockEntries;
+    uint32_t *s_bmx = reinterpret_cast<uint32_t *>(smem) + kRouteWarps * kBlockEntries * 4 +
+                      (threadIdx.x >> 5) * kBlockEntries;
+    // bias of expert sl * EPL + q at s_bias[q * LPT + sl] (lanes of a token read neighbouring words),
+    // zero past E; then 16 words of availability bits, bit e = expert e has a live replica
+    constexpr int kBiasWords = (EPL + 3) / 4 * 4 * 16;
+    float *s_bias = reinterpret_cast<float *>(smem) + kRouteWarps * kBlockEntries * 5;
+    uint32_t *s_avail = reinterpret_cast<uint32_t *>(s_bias + kBiasWords);               // [16]
+    int32_t *s_live = smem + kRouteWarps * kBlockEntries * 5 + kBiasWords + 16;   // [E][1 + max_rep] live count, live slots
     int32_t *s_slot = s_live + E * live_words;        // [NA] slot of each assignment of the tile
     int32_t *s_lrank = s_slot + NA;                   // [NA] stable rank inside the tile
     int32_t *s_hist = s_lrank + NA;                   // [p_pad] tile histogram (running)
@@ -289,7 +296,11 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
     const unsigned full = 0xffffffffu;
 
     // Before the wait only this CTA's own shared memory is touched.
+    // (Loops that a thread passes through about once are kept rolled throughout this kernel: it
+    // is paced by instruction fetch, and unrolled copies of once-run code only add to that.)
+#pragma unroll 1
     for (int q = tid; q < p.p_pad; q += kRouteThreads) { s_hist[q] = 0; s_excl[q] = 0; }
+#pragma unroll 1
     for (int q = tid; q < kRouteWarps * P; q += kRouteThreads) s_wcount[q] = 0;
 
     // Wait for the previous kernel first and only then let the scatter be scheduled: the scatter
@@ -305,8 +316,19 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
         s_epoch = (unsigned)(te >> 32);
     }
     // live replica lists (availability mask and replica pick) and the layout order of the slots
+#pragma unroll 1
     for (int i = tid; i < E * live_words; i += kRouteThreads) s_live[i] = p.live[i];
+    if (tid < 512) {                                   // E <= 512: whole warps, one expert per thread
+        const bool live = tid < E && p.live[tid * live_words] > 0;
+        const unsigned bits = __ballot_sync(full, live);
+        if (lane == 0) s_avail[tid >> 5] = bits;       // all 16 words are written, zero past E
+    }
+    if (tid < kBiasWords) {                            // every word of the table has this one writer
+        const int q = tid / LPT, e = (tid % LPT) * EPL + q;
+        s_bias[tid] = (p.score_func == 1 && q < EPL && e < E) ? p.bias[e] : 0.0f;
+    }
     const int32_t *order = p.state + kStateHeaderWords + p.rank_words + p.expert_words + E * p.max_rep;
+#pragma unroll 1
     for (int q = tid; q < P; q += kRouteThreads) s_order[q] = order[q];
     const int fallback_expert = p.state[0];
     __syncthreads();
@@ -325,11 +347,13 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
     // which of this lane's experts have a live replica: the same for every token it routes
     constexpr int kTokPerWarp = 32 / LPT;
     const int sub = lane / LPT, sl = lane % LPT;
-    uint32_t avail_mask = 0;
-#pragma unroll
-    for (int q = 0; q < EPL; ++q) {
-        const int e = sl * EPL + q;
-        if (e < E && s_live[e * live_words] > 0) avail_mask |= 1u << q;
+    uint32_t avail_mask;
+    {
+        const int e0 = sl * EPL;                          // EPL <= 32 bits starting at bit e0 of the bitmap
+        const uint32_t lo = s_avail[(e0 >> 5) & 15], hi = s_avail[((e0 >> 5) + 1) & 15];
+        avail_mask = __funnelshift_r(lo, hi, e0 & 31);
+        avail_mask &= 0xffffffffu >> (32 - EPL);
+        if (e0 >= E) avail_mask = 0;
     }
 
     // Dense-FFN mode (score_func 2): the "experts" are the k = TP shards of E/k replicated
@@ -338,8 +362,10 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
     if (dense) {
         if (tid == 0) {
             int n = 0;
+#pragma unroll 1
             for (int g = 0; g < E / k; ++g) {
                 bool healthy = true;
+#pragma unroll 1
                 for (int sh = 0; sh < k; ++sh) healthy = healthy && (s_live[(g * k + sh) * live_words] > 0);
                 if (healthy) s_lrank[n++] = g;             // s_lrank is free until the histogram step
             }
@@ -350,6 +376,7 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
     const int n_healthy = dense ? s_warp_sums[0] : 0;
 
     // ---- gate, mask, selection, weights, replica: per token ----------------
+#pragma unroll 1
     for (int lt0 = warp * kTokPerWarp; lt0 < tb; lt0 += kRouteWarps * kTokPerWarp) {
         const int lt = lt0 + sub;
         const int t = t0 + lt;
@@ -364,7 +391,8 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
                     slot = s_live[id * live_words + 1 + t % s_live[id * live_words]];
                 }
             } else {
-                route_tokens<EPL, LPT>(p, t0 + lt0, avail_mask, s_live, fallback_expert, id, w, slot);
+                route_tokens<EPL, LPT>(p, t0 + lt0, avail_mask, s_live, s_bias, s_blk, s_bmx, fallback_expert,
+                                       id, w, slot);
             }
             if (t >= p.T) slot = -1;
             if (sl < k && t < p.T) {
@@ -382,6 +410,7 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
     // Rounds of 1024 assignments in ascending i.  Inside a round, match_any gives
     // the rank among equal slots of a warp and the per-warp counts; a scan down
     // each slot's column of counts orders the warps.
+#pragma unroll 1
     for (int base = 0; base < NA; base += kRouteThreads) {
         const int i = base + tid;
         const int slot = (i < NA) ? s_slot[i] : -1;
@@ -389,9 +418,10 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
         const int rank_in_warp = __popc(peers & lanemask_lt());
         if (slot >= 0 && rank_in_warp == 0) s_wcount[warp * P + slot] = (uint16_t)__popc(peers);
         __syncthreads();
+#pragma unroll 1
         for (int q = tid; q < P; q += kRouteThreads) {
             int run = s_hist[q];
-#pragma unroll 8
+#pragma unroll 4
             for (int w2 = 0; w2 < kRouteWarps; ++w2) {
                 const int c = s_wcount[w2 * P + q];
                 s_wcount[w2 * P + q] = (uint16_t)run;      // run < 65536: a tile has <= 32768 assignments
@@ -403,6 +433,7 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
         if (slot >= 0) s_lrank[i] = (int)s_wcount[warp * P + slot] + rank_in_warp;
         if (base + kRouteThreads < NA) {
             __syncthreads();
+#pragma unroll 1
             for (int q = tid; q < kRouteWarps * P; q += kRouteThreads) s_wcount[q] = 0;
             __syncthreads();
         }
@@ -413,6 +444,7 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
     {
         ulonglong2 *mine = p.tile_counts + (size_t)ticket * groups;
         const unsigned long long tag = (unsigned long long)epoch << 32;
+#pragma unroll 1
         for (int q4 = tid; q4 < groups; q4 += kRouteThreads) {
             const int32_t *h = s_hist + 4 * q4;            // entries past P stay zero
             st_relaxed_v2_u64(mine + q4, tag | (unsigned)h[0] | ((unsigned)h[1] << 16),
@@ -429,7 +461,8 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
             // Up to kBatch entries are requested together and the stale ones (their tile has not
             // published yet) are requested again together, so a round of retries costs one trip
             // to L2 however many of the entries were stale.
-            constexpr int kBatch = 6;
+            constexpr int kBatch = 4;
+#pragma unroll 1
             for (int b0 = g; b0 < (int)ticket && !gave_up; b0 += nseg * kBatch) {
                 ulonglong2 v[kBatch];
                 unsigned pending = 0;
@@ -483,6 +516,7 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
     }
 
     // stable rank of every assignment of the tile inside its slot, over all tiles
+#pragma unroll 1
     for (int i = tid; i < n_tok * k; i += kRouteThreads)
         p.pos_in_slot[(size_t)t0 * k + i] = s_excl[s_slot[i]] + s_lrank[i];
 
@@ -491,11 +525,13 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
     // ---- the last tile knows every total: per-slot counts and offsets -----
     // exclusive scan over the P layout positions (position q holds physical slot order[q]),
     // a contiguous chunk of positions per thread
+#pragma unroll 1
     for (int q = tid; q < P; q += kRouteThreads) s_hist[q] += s_excl[q];     // totals per physical slot
     __syncthreads();
     const int chunk = (P + kRouteThreads - 1) / kRouteThreads;
     const int q0 = tid * chunk;
     int local = 0;
+#pragma unroll 1
     for (int q = q0; q < min(P, q0 + chunk); ++q) local += s_hist[s_order[q]];
     int incl = local;
     for (int off = 1; off < 32; off <<= 1) {
@@ -505,8 +541,10 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
     if (lane == 31) s_warp_sums[warp] = incl;
     __syncthreads();                                   // also: all reads of s_excl above are done
     int warp_base = 0;
+#pragma unroll 1
     for (int w2 = 0; w2 < warp; ++w2) warp_base += s_warp_sums[w2];
     int run = warp_base + incl - local;
+#pragma unroll 1
     for (int q = q0; q < min(P, q0 + chunk); ++q) {
         const int slot = s_order[q];
         const int tot = s_hist[slot];
@@ -520,8 +558,10 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
         p.rank_offsets[p.R] = run;
     }
     __syncthreads();
+#pragma unroll 1
     for (int r = tid; r < p.R; r += kRouteThreads) {   // r-th rank of the layout order
         int c = 0;
+#pragma unroll 1
         for (int s = 0; s < p.S; ++s) c += s_hist[s_order[r * p.S + s]];
         p.rank_counts[r] = c;
         p.rank_offsets[r] = s_excl[r * p.S];

@@ -14,9 +14,19 @@ module only wires the pieces together:
 """
 from __future__ import annotations
 
-import torch
+import os
 
-from . import binding as B
+# The receive buffers are reached with plain peer loads, stores and (non-multicast) bulk
+# copies only, so they are never bound to an NVLink multicast object, and the collectives
+# used here (an all-gather of a few KB, one-word all-reduces) gain nothing from in-switch
+# reduction.  Both libraries read these settings when they initialise, so they are set
+# on import, before the caller creates its process group; a caller's own setting wins.
+os.environ.setdefault("TORCH_SYMM_MEM_DISABLE_MULTICAST", "1")
+os.environ.setdefault("NCCL_NVLS_ENABLE", "0")
+
+import torch  # noqa: E402
+
+from . import binding as B  # noqa: E402
 
 
 def gather_counts(slot_counts: torch.Tensor, group=None) -> torch.Tensor:

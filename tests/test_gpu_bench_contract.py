@@ -19,7 +19,8 @@ def test_bench_prints_one_json_line_with_every_key():
     r = json.loads(lines[0])
     for key in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better",
                 "scaling", "vs_baseline", "dtype", "data", "config", "clocks", "e2e", "gpu_launches",
-                "roofline", "cpu_baseline", "remap"):
+                "roofline", "cpu_baseline", "remap", "timed_repeats", "ms_per_step_min", "ms_per_step_max",
+                "kimi_remap_sweep"):
         assert key in r, key
     assert r["value"] > 0 and r["steps"] == 20 and r["n_gpus"] == 1 and r["scaling"] == "weak"
     assert r["vs_baseline"] is None and r["data"] == "synthetic" and "workload" in r["config"]
@@ -28,5 +29,9 @@ def test_bench_prints_one_json_line_with_every_key():
     assert rf["bound"] == "hbm" and rf["unit"] == "GB/s" and abs(rf["frac"] - rf["achieved"] / rf["peak"]) < 1e-9
     assert rf["traffic"] is None                       # ncu traffic figures belong to the DSv3 shape only
     assert r["cpu_baseline"]["kind"] == "oracle" and r["cpu_baseline"]["cores"] == 1
+    assert r["cpu_baseline"]["host_cores"] >= 1 and "cpu_model" in r["cpu_baseline"]
+    assert r["timed_repeats"] >= 3 and r["clocks"]["samples"] >= 5
+    assert r["kimi_remap_sweep"] is None               # part of the default (DSv3-shaped) run only
+    assert "eager leg" in rf["per_kernel_source"]
     assert r["e2e"]["h2d_bytes_per_step"] > 0 and r["e2e"]["d2h_bytes_per_step"] > 0
     assert r["remap"]["first_step_matches_oracle"] is True and r["remap"]["graph_recaptured"] is False

@@ -1,7 +1,7 @@
-"""World-size-2 check (gloo, CPU) of the host logic the multi-GPU benchmark
-uses: every rank draws its own batch and the step time is the maximum over
-ranks.  The data path itself has no collective: ranks route independent
-batches (weak scaling)."""
+"""World-size-2 checks (gloo, CPU) of the host logic the multi-GPU benchmark uses: the step
+time is the maximum over ranks, replicas draw their own batches, and `bench.py --gpus 2`
+starts two ranks by itself, shards tokens and slots, exchanges the per-slot counts and
+prints one JSON line (walked here with `--dry-run`, which touches no GPU)."""
 import os
 import socket
 import subprocess
@@ -73,3 +73,30 @@ def test_reference_arm_prints_one_json_line():
     rec = json.loads(lines[0])
     assert rec["impl"] == "reference" and rec["value"] > 0 and rec["cpu_baseline"]["kind"] == "oracle"
     assert rec["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def test_bench_starts_its_own_ranks_and_prints_one_line():
+    import json
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--dry-run",
+                          "--steps", "5", "--warmup", "3"],
+                         capture_output=True, text=True, timeout=600, cwd=ROOT,
+                         env={k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")})
+    assert out.returncode == 0, out.stdout[-2000:] + out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.strip().startswith("{")]
+    assert len(lines) == 1, out.stdout
+    rec = json.loads(lines[0])
+    assert rec["dry_run"] is True and rec["n_gpus"] == 2 and rec["scaling"] == "strong"
+    assert rec["config"]["T_per_gpu"] == 4096 and rec["config"]["slots_per_gpu"] == 144
+    assert rec["rows_total"] == 8192 * 8 and rec["max_over_ranks_check"] == 2.0
+    for key in ("metric", "unit", "steps", "warmup", "higher_is_better", "vs_baseline", "dtype", "data", "config"):
+        assert key in rec, key
+
+
+def test_token_shards_cover_the_batch():
+    import bench
+    for T, world in ((8192, 8), (10, 4), (3, 8), (0, 2)):
+        spans = [bench.shard_tokens(T, world, r) for r in range(world)]
+        assert spans[0][0] == 0 and spans[-1][1] == T
+        assert all(a[1] == b[0] for a, b in zip(spans, spans[1:]))
+        sizes = [hi - lo for lo, hi in spans]
+        assert max(sizes) - min(sizes) <= 1
