@@ -310,30 +310,33 @@ def remap_leg(router, graph, out, wl, inp, sets, restore, n_iter=30):
     for fs in set(sets):
         ref = oracle_reference_outputs(wl, inp, fs, with_bias)
         refs[fs] = {f: torch.from_numpy(np.ascontiguousarray(ref[f]).reshape(-1)).to(dev) for f in INT_FIELDS}
-    steady, with_remap, host_us, ok = [], [], [], True
-    for _ in range(n_iter):
+    steady, added, host_us, ok = [], [], [], True
+    for i in range(n_iter):
+        # a plain replay and a remap + replay back to back, so that slow drift of the step time
+        # cancels in their difference
+        fs = sets[i % len(sets)]
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         graph.replay()
         torch.cuda.synchronize()
-        steady.append(time.perf_counter() - t0)
-    for i in range(n_iter):
-        fs = sets[i % len(sets)]
-        torch.cuda.synchronize()
+        t_plain = time.perf_counter() - t0
         t0 = time.perf_counter()
         router.set_failed_ranks(fs)
         t1 = time.perf_counter()
         graph.replay()
         torch.cuda.synchronize()
-        with_remap.append(time.perf_counter() - t0)
+        t_remap = time.perf_counter() - t0
+        steady.append(t_plain)
+        added.append(t_remap - t_plain)
         host_us.append((t1 - t0) * 1e6)
         ok = ok and matches_oracle(out, refs[fs])     # outside the timed part
     router.set_failed_ranks(restore)
     return {"host_call_us_median": statistics.median(host_us),
-            "added_latency_us_median": (statistics.median(with_remap) - statistics.median(steady)) * 1e6,
+            "added_latency_us_median": statistics.median(added) * 1e6,
             "step_us_median": statistics.median(steady) * 1e6,
             "first_step_matches_oracle": bool(ok),
             "checked": "every first step after a remap: " + ", ".join(INT_FIELDS),
+            "added_latency": "median over pairs of (remap + replay + sync) - (replay + sync), wall clock",
             "failure_sets_cycled": [list(s) for s in sets], "launches": 3 * 2 * n_iter + n_iter}
 
 
@@ -376,30 +379,28 @@ def kimi_remap_sweep(dev, steps=20):
             first = time.perf_counter() - t0
             ok = matches_oracle(out, ref_dev)
             no_failed_rows = bool((out.rank_counts[list(fs)] == 0).all()) if fs else True
-            steady, with_remap = [], []
-            for _ in range(7):
+            added = []
+            for _ in range(9):                           # plain replay, then remap + replay: the difference
                 torch.cuda.synchronize()
                 t0 = time.perf_counter()
                 graph.replay()
                 torch.cuda.synchronize()
-                steady.append(time.perf_counter() - t0)
-            for _ in range(7):
-                torch.cuda.synchronize()
+                t_plain = time.perf_counter() - t0
                 t0 = time.perf_counter()
                 router.set_failed_ranks(fs)
                 graph.replay()
                 torch.cuda.synchronize()
-                with_remap.append(time.perf_counter() - t0)
+                added.append(time.perf_counter() - t0 - t_plain)
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(stream)
             for _ in range(steps):
                 graph.replay()
             e1.record(stream)
             torch.cuda.synchronize()
-            launches += 3 * (15 + steps) + 8
+            launches += 3 * (19 + steps) + 10
             rows.append({"failed_ranks": n, "first_step_matches_oracle": bool(ok),
                          "failed_ranks_own_no_rows": no_failed_rows,
-                         "added_latency_us": (statistics.median(with_remap) - statistics.median(steady)) * 1e6,
+                         "added_latency_us": statistics.median(added) * 1e6,
                          "first_step_us_wall": first * 1e6,
                          "steady_tokens_per_s": T * steps / (e0.elapsed_time(e1) * 1e-3),
                          "steady_us_per_step": e0.elapsed_time(e1) * 1e3 / steps})
@@ -408,8 +409,8 @@ def kimi_remap_sweep(dev, steps=20):
     return {"workload": workload_name(wl, ()), "tokens": T, "graph_captures": captures,
             "graph_recaptured": captures != 1, "rows": rows,
             "what": "full Kimi-K2 shape; per failed-rank count: remap + first replay of the one captured graph "
-                    "checked against the oracle (" + ", ".join(INT_FIELDS) + "), added latency = median wall "
-                    "time of remap+replay minus median replay, steady throughput over "
+                    "checked against the oracle (" + ", ".join(INT_FIELDS) + "), added latency = median over 9 pairs "
+                    "of (wall time of remap + replay) - (wall time of the replay before it), steady throughput over "
                     f"{steps} replays (CUDA events)", "launches": launches}
 
 

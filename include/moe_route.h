@@ -344,7 +344,9 @@ typedef enum {
     MOE_TUNE_COMBINE_CTAS_PER_SM = 10,    /* ring combine: CTAs per SM (default: as many as fit)                 */
     MOE_TUNE_ROUTE_LANES_PER_TOKEN = 11,  /* routing: 8 or 16 lanes of a warp per token                          */
     MOE_TUNE_ROUTE_TOKENS_PER_TILE = 12,  /* routing: tokens per tile (default: max_tokens / 148, at least 32)   */
-    MOE_TUNE_SPIN_LIMIT = 13              /* polls before a bounded device wait gives up (default 1 << 20)       */
+    MOE_TUNE_SPIN_LIMIT = 13,             /* polls before a bounded device wait gives up (default 1 << 20)       */
+    MOE_TUNE_ROUTE_PREFETCH = 14          /* routing: L2 hints issued while the previous kernel drains; bit 0 the
+                                             routing tables, bit 1 the logits (default 3)                        */
 } moe_tuning_option;
 
 moe_status moe_set_tuning(moe_ctx *ctx, int32_t option, int32_t value);

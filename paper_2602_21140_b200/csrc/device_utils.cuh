@@ -65,6 +65,12 @@ __device__ __forceinline__ int ld_relaxed_s32(const int *p)
     return v;
 }
 
+// Hint: pull the cache line holding *p into L2.
+__device__ __forceinline__ void prefetch_l2(const void *p)
+{
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+}
+
 // Asynchronous copies global -> shared that bypass registers; wait_all covers the calling
 // thread's own copies (enough when the same thread reads what it asked for).
 __device__ __forceinline__ void cp_async_16(void *smem_dst, const void *gsrc)

@@ -28,7 +28,7 @@ constexpr int kMaxSlots = 4096;
 constexpr int kStagingSlots = 16;
 constexpr size_t kMaxSmem = 227 * 1024;
 constexpr int kRouteTileTarget = 148;   // tiles of a full step: one per SM of a B200
-constexpr int kNumTuning = MOE_TUNE_SPIN_LIMIT + 1;
+constexpr int kNumTuning = MOE_TUNE_ROUTE_PREFETCH + 1;
 
 // Shape-derived launch constants.
 struct Derived {
@@ -111,6 +111,8 @@ bool derive(const moe_config *c, Derived *d, int want_lpt = 0, int want_tile = 0
     // routes at once.  Halved until the tile's tables fit in shared memory.
     const int per_warp = 32 / d->lpt;
     int tile = want_tile > 0 ? want_tile : std::max(32, (c->max_tokens + kRouteTileTarget - 1) / kRouteTileTarget);
+    // a batch that one CTA routes in a single pass of its 32 warps needs no prefix over tiles at all
+    if (want_tile <= 0 && c->max_tokens <= kRouteWarps * per_warp) tile = c->max_tokens;
     tile = (tile + per_warp - 1) / per_warp * per_warp;
     while (tile > per_warp &&
            (route_smem_bytes(d->E, d->max_rep, tile, d->k, d->P, d->epl) > kMaxSmem - 1024 || (long long)tile * d->k > 65535))
@@ -234,6 +236,7 @@ struct moe_ctx {
     int scatter_impl;      // 0 = vector, 1 = bulk copies
     int bulk_stages, bulk_ctas_per_sm;
     int scatter_blocks_per_sm, combine_blocks_per_sm, scatter_unroll;
+    int route_prefetch;    // L2 hints issued by the routing kernel before its wait (bit 0 tables, bit 1 logits)
     int combine_impl;      // 0 = vector loads, 1 = bulk-copy ring
     int combine_stages, combine_u, combine_ctas_per_sm, combine_warps;
     size_t combine_smem;
@@ -357,6 +360,7 @@ cudaError_t enqueue_route(moe_ctx *ctx, const float *logits, int32_t T, const mo
     rp.slot_counts = out->slot_counts; rp.slot_offsets = out->slot_offsets;
     rp.rank_counts = out->rank_counts; rp.rank_offsets = out->rank_offsets;
     rp.tile_counts = ctx->d_tile_counts; rp.ctl = ctx->d_ctl;
+    rp.prefetch = ctx->pdl ? ctx->route_prefetch : 0;
     const int tiles = (T + d.tokens_per_block - 1) / d.tokens_per_block;
     return launch_route(d.epl, d.lpt, rp, tiles, ctx->route_smem, st, ctx->pdl);
 }
@@ -495,10 +499,16 @@ void configure_launch(moe_ctx *ctx)
         const int need = (d.H / 8 + 31) / 32;
         int un = 32;
         for (int u : kUnroll) if (u >= need) { un = u; break; }
+        // ... unless the whole scatter is short (under 256 MB moved, a few tens of microseconds):
+        // then the start-up of each warp's single long copy is not amortised and 2 KB pieces,
+        // four times as many warps' worth of work, win (33.4 against 35.0 us per step at 4096
+        // tokens of 8 KB; at 8192 tokens of 14 KB whole rows are 3 % of a step faster)
+        if ((long long)ctx->cfg.max_tokens * d.H * 2 * (1 + d.k) < (256ll << 20)) un = 4;
         const int forced = tuned(ctx, MOE_TUNE_SCATTER_UNROLL, 0);
         for (int u : kUnroll) if (u == forced) un = forced;
         ctx->scatter_unroll = un;
     }
+    ctx->route_prefetch = tuned(ctx, MOE_TUNE_ROUTE_PREFETCH, 3) & 3;
     ctx->combine_blocks_per_sm = 8;
     ctx->combine_impl = tuned(ctx, MOE_TUNE_COMBINE_IMPL, 1);
     // a ring stage holds one column chunk of all k rows: widen the chunk for small k so that a

@@ -89,6 +89,7 @@ struct RouteParams {
     int32_t *topk_slot;       // [T,k]
     int32_t *pos_in_slot;     // [T*k]: stable rank of assignment i inside its slot
     int32_t *slot_counts, *slot_offsets, *rank_counts, *rank_offsets;
+    int prefetch;             // bit 0: ask the small tables into L2 before the wait; bit 1: the logits too
     ulonglong2 *tile_counts;  // [tiles][p_pad/4]: per tile, four slots to a 16-byte entry: two words
                               // of (epoch << 32 | count of the odd slot << 16 | count of the even slot)
     Control *ctl;
@@ -303,6 +304,28 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
 #pragma unroll 1
     for (int q = tid; q < kRouteWarps * P; q += kRouteThreads) s_wcount[q] = 0;
 
+    // ... apart from hints: under programmatic dependent launch this CTA may be resident well
+    // before the previous kernel has finished, and the tables it is about to read were last
+    // touched a whole step ago (2 GB of rows have passed through L2 since).  Asking for them now
+    // turns DRAM misses on the critical path into L2 hits.  A hint cannot return stale data:
+    // L2 is where every write lands.
+    if (p.prefetch & 1) {
+        const int words = E * live_words;
+        if (tid * 32 < words) prefetch_l2(p.live + tid * 32);
+        if (tid * 32 < P) prefetch_l2(p.state + kStateHeaderWords + p.rank_words + p.expert_words + E * p.max_rep + tid * 32);
+        if (tid * 32 < E) prefetch_l2(p.bias + tid * 32);
+        if (tid == 0) { prefetch_l2(p.ctl); prefetch_l2(p.state); }
+    }
+    if ((p.prefetch & 2) && p.logits != nullptr) {
+        // the tile is not known before the ticket: every CTA asks for an equal share of the tensor
+        const size_t total = (size_t)p.T * E * sizeof(float);
+        const size_t share = ((total + gridDim.x - 1) / gridDim.x + 127) & ~(size_t)127;
+        const size_t lo = (size_t)blockIdx.x * share, hi = min(total, lo + share);
+#pragma unroll 1
+        for (size_t off = lo + (size_t)tid * 128; off < hi; off += (size_t)kRouteThreads * 128)
+            prefetch_l2(reinterpret_cast<const char *>(p.logits) + off);
+    }
+
     // Wait for the previous kernel first and only then let the scatter be scheduled: the scatter
     // requests its first x rows before its own wait, which is safe only once whatever produced x
     // (a kernel before this one) is known to have completed.
@@ -461,7 +484,7 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
             // Up to kBatch entries are requested together and the stale ones (their tile has not
             // published yet) are requested again together, so a round of retries costs one trip
             // to L2 however many of the entries were stale.
-            constexpr int kBatch = 4;
+            constexpr int kBatch = 8;
 #pragma unroll 1
             for (int b0 = g; b0 < (int)ticket && !gave_up; b0 += nseg * kBatch) {
                 ulonglong2 v[kBatch];
