@@ -52,7 +52,7 @@ MIN_TIMED_SECONDS = 0.3          # the timed region is repeated until it spans a
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from ncu captures of
 # the kernels as they stand at the DSv3 shape (summaries under profiles/); None when a kernel
 # changed after its last capture.
-NCU_TRAFFIC_BYTES = {"k_scatter": None, "k_combine": None}
+NCU_TRAFFIC_BYTES = {"k_scatter": 998_396_160, "k_combine": 1_051_368_192}
 
 INT_FIELDS = ("topk_ids", "topk_slot", "slot_counts", "slot_offsets", "rank_counts", "rank_offsets", "dst_row")
 

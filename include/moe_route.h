@@ -345,8 +345,11 @@ typedef enum {
     MOE_TUNE_ROUTE_LANES_PER_TOKEN = 11,  /* routing: 8 or 16 lanes of a warp per token                          */
     MOE_TUNE_ROUTE_TOKENS_PER_TILE = 12,  /* routing: tokens per tile (default: max_tokens / 148, at least 32)   */
     MOE_TUNE_SPIN_LIMIT = 13,             /* polls before a bounded device wait gives up (default 1 << 20)       */
-    MOE_TUNE_ROUTE_PREFETCH = 14          /* routing: L2 hints issued while the previous kernel drains; bit 0 the
+    MOE_TUNE_ROUTE_PREFETCH = 14,         /* routing: L2 hints issued while the previous kernel drains; bit 0 the
                                              routing tables, bit 1 the logits (default 3)                        */
+    MOE_TUNE_SCATTER_STORE_POLICY = 15    /* vector scatter, pieces of 4, 16 or 28 units: cache policy of the row
+                                             stores; 0 (default) no L1 allocation, 1 plain, 2 L2 evict-first,
+                                             3 streaming                                                         */
 } moe_tuning_option;
 
 moe_status moe_set_tuning(moe_ctx *ctx, int32_t option, int32_t value);

@@ -39,7 +39,7 @@ MOE_ROUTE_DENSE_TP = 2
  MOE_TUNE_SCATTER_BLOCKS_PER_SM, MOE_TUNE_SCATTER_UNROLL, MOE_TUNE_COMBINE_IMPL, MOE_TUNE_COMBINE_CHUNK,
  MOE_TUNE_COMBINE_STAGES, MOE_TUNE_COMBINE_WARPS, MOE_TUNE_COMBINE_CTAS_PER_SM,
  MOE_TUNE_ROUTE_LANES_PER_TOKEN, MOE_TUNE_ROUTE_TOKENS_PER_TILE, MOE_TUNE_SPIN_LIMIT,
- MOE_TUNE_ROUTE_PREFETCH) = range(15)
+ MOE_TUNE_ROUTE_PREFETCH, MOE_TUNE_SCATTER_STORE_POLICY) = range(16)
 
 EXPORTED_SYMBOLS = (
     "moe_route_init", "moe_set_failed_ranks", "moe_update_replica_map", "moe_dispatch",

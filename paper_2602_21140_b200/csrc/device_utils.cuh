@@ -110,6 +110,32 @@ __device__ __forceinline__ void st_stream_v4(uint4 *p, const uint4 &v)
                  : "memory");
 }
 
+// The same store with another cache policy, for measurements of what the write policy of the
+// scatter does to the kernel that follows it: 1 = plain store, 2 = L2 evict-first hint,
+// 3 = streaming (.cs) store.  0 is st_stream_v4.
+__device__ __forceinline__ unsigned long long l2_policy_evict_first()
+{
+    unsigned long long pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+
+template <int POLICY>
+__device__ __forceinline__ void st_policy_v4(uint4 *p, const uint4 &v, unsigned long long pol)
+{
+    if (POLICY == 1) {
+        asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+    } else if (POLICY == 2) {
+        asm volatile("st.global.L1::no_allocate.L2::cache_hint.v4.u32 [%0], {%1,%2,%3,%4}, %5;" ::"l"(p), "r"(v.x),
+                     "r"(v.y), "r"(v.z), "r"(v.w), "l"(pol)
+                     : "memory");
+    } else if (POLICY == 3) {
+        asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+    } else {
+        st_stream_v4(p, v);
+    }
+}
+
 // ---------------------------------------------------------------------------
 // exp / sigmoid from single IEEE fp32 operations (round to nearest even, never
 // contracted, independent of compiler flags), so that sigmoid routing keys are

@@ -28,7 +28,7 @@ constexpr int kMaxSlots = 4096;
 constexpr int kStagingSlots = 16;
 constexpr size_t kMaxSmem = 227 * 1024;
 constexpr int kRouteTileTarget = 148;   // tiles of a full step: one per SM of a B200
-constexpr int kNumTuning = MOE_TUNE_ROUTE_PREFETCH + 1;
+constexpr int kNumTuning = MOE_TUNE_SCATTER_STORE_POLICY + 1;
 
 // Shape-derived launch constants.
 struct Derived {
@@ -236,6 +236,7 @@ struct moe_ctx {
     int scatter_impl;      // 0 = vector, 1 = bulk copies
     int bulk_stages, bulk_ctas_per_sm;
     int scatter_blocks_per_sm, combine_blocks_per_sm, scatter_unroll;
+    int scatter_store_policy;   // 0 = default (no L1 allocation); 1 plain, 2 L2 evict-first, 3 streaming
     int route_prefetch;    // L2 hints issued by the routing kernel before its wait (bit 0 tables, bit 1 logits)
     int combine_impl;      // 0 = vector loads, 1 = bulk-copy ring
     int combine_stages, combine_u, combine_ctas_per_sm, combine_warps;
@@ -508,6 +509,13 @@ void configure_launch(moe_ctx *ctx)
         for (int u : kUnroll) if (u == forced) un = forced;
         ctx->scatter_unroll = un;
     }
+    // Row stores normally skip L1 and leave L2 early (the rows are read again only after ~1 GB of
+    // other rows has passed).  A send buffer small enough to stay in the 126 MB L2 until the
+    // combine reads it is written with plain stores instead: 31.8 against 33.7 us per step at 4096
+    // tokens of 8 KB, k = 2 (67 MB); at 940 MB plain stores cost 4 us.
+    const bool fits_l2 = (long long)ctx->cfg.max_tokens * d.k * d.H * 2 <= (80ll << 20);
+    ctx->scatter_store_policy = std::min(3, tuned(ctx, MOE_TUNE_SCATTER_STORE_POLICY, fits_l2 ? 1 : 0));
+    if (ctx->scatter_unroll != 28 && ctx->scatter_unroll != 16 && ctx->scatter_unroll != 4) ctx->scatter_store_policy = 0;
     ctx->route_prefetch = tuned(ctx, MOE_TUNE_ROUTE_PREFETCH, 3) & 3;
     ctx->combine_blocks_per_sm = 8;
     ctx->combine_impl = tuned(ctx, MOE_TUNE_COMBINE_IMPL, 1);
@@ -828,12 +836,25 @@ moe_status moe_dispatch(moe_ctx *ctx, const float *logits, const void *x, int32_
         const long long items = (long long)T * chunks;
         const long long want = (items + kScatterThreads / 32 - 1) / (kScatterThreads / 32);
         const int grid = (int)std::min<long long>(want, (long long)ctx->sm_count * ctx->scatter_blocks_per_sm);
-        switch (un) {
-            case 8: launch_kernel(k_scatter_vec<8>, dim3(grid), dim3(kScatterThreads), 0, st, ctx->pdl, sp); break;
-            case 16: launch_kernel(k_scatter_vec<16>, dim3(grid), dim3(kScatterThreads), 0, st, ctx->pdl, sp); break;
-            case 28: launch_kernel(k_scatter_vec<28>, dim3(grid), dim3(kScatterThreads), 0, st, ctx->pdl, sp); break;
-            case 32: launch_kernel(k_scatter_vec<32>, dim3(grid), dim3(kScatterThreads), 0, st, ctx->pdl, sp); break;
-            default: launch_kernel(k_scatter_vec<4>, dim3(grid), dim3(kScatterThreads), 0, st, ctx->pdl, sp); break;
+        const dim3 g(grid), b(kScatterThreads);
+        const bool pdl = ctx->pdl;
+        switch (un * 10 + ctx->scatter_store_policy) {
+            case 80: launch_kernel(k_scatter_vec<8, 0>, g, b, 0, st, pdl, sp); break;
+            case 160: launch_kernel(k_scatter_vec<16, 0>, g, b, 0, st, pdl, sp); break;
+            case 280: launch_kernel(k_scatter_vec<28, 0>, g, b, 0, st, pdl, sp); break;
+            case 320: launch_kernel(k_scatter_vec<32, 0>, g, b, 0, st, pdl, sp); break;
+            case 40: launch_kernel(k_scatter_vec<4, 0>, g, b, 0, st, pdl, sp); break;
+            // the other store policies: measurement variants of the two most used shapes
+            case 281: launch_kernel(k_scatter_vec<28, 1>, g, b, 0, st, pdl, sp); break;
+            case 282: launch_kernel(k_scatter_vec<28, 2>, g, b, 0, st, pdl, sp); break;
+            case 283: launch_kernel(k_scatter_vec<28, 3>, g, b, 0, st, pdl, sp); break;
+            case 161: launch_kernel(k_scatter_vec<16, 1>, g, b, 0, st, pdl, sp); break;
+            case 162: launch_kernel(k_scatter_vec<16, 2>, g, b, 0, st, pdl, sp); break;
+            case 163: launch_kernel(k_scatter_vec<16, 3>, g, b, 0, st, pdl, sp); break;
+            case 41: launch_kernel(k_scatter_vec<4, 1>, g, b, 0, st, pdl, sp); break;
+            case 42: launch_kernel(k_scatter_vec<4, 2>, g, b, 0, st, pdl, sp); break;
+            case 43: launch_kernel(k_scatter_vec<4, 3>, g, b, 0, st, pdl, sp); break;
+            default: return MOE_ERR_INVALID_ARG;          // policy not built for this piece size
         }
     }
     if (cudaGetLastError() != cudaSuccess) return MOE_ERR_CUDA;

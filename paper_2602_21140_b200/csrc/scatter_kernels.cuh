@@ -53,7 +53,9 @@ __device__ __forceinline__ int resolve_row(const ScatterParams &p, int t, int la
 }
 
 // UNROLL = 16-byte loads in flight per lane; a work item is 32*UNROLL 16-byte units of a row.
-template <int UNROLL>
+// POLICY = cache policy of the stores (0, the default: no L1 allocation; the others exist to
+// measure what the write policy does to the combine that follows, see st_policy_v4).
+template <int UNROLL, int POLICY = 0>
 __global__ void __launch_bounds__(kScatterThreads) k_scatter_vec(ScatterParams p)
 {
     constexpr int kChunk = 32 * UNROLL;
@@ -65,6 +67,7 @@ __global__ void __launch_bounds__(kScatterThreads) k_scatter_vec(ScatterParams p
     const long long warp0 = (long long)blockIdx.x * (kScatterThreads / 32) + (threadIdx.x >> 5);
     const long long nwarps = (long long)gridDim.x * (kScatterThreads / 32);
 
+    const unsigned long long pol = (POLICY == 2) ? l2_policy_evict_first() : 0ull;
     bool waited = false;
     for (long long it = warp0; it < items; it += nwarps) {
         const int t = (int)(it / chunks);
@@ -88,7 +91,7 @@ __global__ void __launch_bounds__(kScatterThreads) k_scatter_vec(ScatterParams p
             uint4 *dst = p.send + (size_t)r * p.hv;
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u)
-                if (c0 + 32 * u < p.hv) st_stream_v4(dst + c0 + 32 * u, v[u]);
+                if (c0 + 32 * u < p.hv) st_policy_v4<POLICY>(dst + c0 + 32 * u, v[u], pol);
         }
     }
 }
