@@ -761,7 +761,15 @@ def run_group(args):
         raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    dist.init_process_group("nccl", device_id=dev)
+    if world == 1:                                      # --exchange on one GPU: a group of one
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        if "MASTER_PORT" not in os.environ:
+            with socket.socket() as s:
+                s.bind(("127.0.0.1", 0))
+                os.environ["MASTER_PORT"] = str(s.getsockname()[1])
+        dist.init_process_group("nccl", device_id=dev, rank=0, world_size=1)
+    else:
+        dist.init_process_group("nccl", device_id=dev)
 
     wl = W.WORKLOADS[args.workload]
     failed = wl.failure_sets[min(args.failure_set, len(wl.failure_sets) - 1)]
@@ -887,7 +895,7 @@ def run_group(args):
         alg = algorithmic_bytes(wl, T)
         print(json.dumps({
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
-            "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "strong",
+            "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "strong" if world > 1 else "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {**base_config(wl, failed), "T_per_gpu": Tl, "slots_per_gpu": wl.P // world,
                        "parallelism": f"ep{world}: tokens sharded T/{world} per GPU, slots P/{world} per GPU; per step "
@@ -1039,6 +1047,8 @@ def main():
     ap.add_argument("--no-kimi-sweep", action="store_true", help="skip the Kimi-K2-shaped remap sweep of the default run")
     ap.add_argument("--tune", action="append", metavar="OPTION=VALUE",
                     help="override a launch choice through moe_set_tuning, e.g. combine_stages=4 (repeatable)")
+    ap.add_argument("--exchange", action="store_true",
+                    help="time the multi-GPU exchange path (moe_ep_*, NCCL) even with one GPU: a group of one")
     ap.add_argument("--dry-run", action="store_true", help="walk the multi-rank protocol on CPU (gloo); no GPU is touched")
     ap.add_argument("--expert-failure-sweep", action="store_true",
                     help="run the lost-expert sweep (throughput and load imbalance against r) instead of the benchmark")
@@ -1054,7 +1064,7 @@ def main():
         return run_expert_failure_sweep(args)
     if args.impl == "reference":
         return run_reference(args)
-    if world > 1:
+    if world > 1 or args.exchange:
         return run_group(args)
     return run_single(args)
 

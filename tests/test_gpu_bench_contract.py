@@ -35,3 +35,19 @@ def test_bench_prints_one_json_line_with_every_key():
     assert "eager leg" in rf["per_kernel_source"]
     assert r["e2e"]["h2d_bytes_per_step"] > 0 and r["e2e"]["d2h_bytes_per_step"] > 0
     assert r["remap"]["first_step_matches_oracle"] is True and r["remap"]["graph_recaptured"] is False
+
+
+@pytest.mark.gpu
+def test_exchange_path_of_the_benchmark_runs_as_a_group_of_one():
+    # the code `bench.py --gpus N` runs on every rank (NCCL, symmetric memory, moe_ep_*), here with N = 1
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--exchange", "--workload", "mixtral",
+                          "--tokens", "512", "--steps", "10", "--warmup", "3"],
+                         capture_output=True, text=True, timeout=900, cwd=ROOT,
+                         env={k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")})
+    assert out.returncode == 0, out.stdout[-1500:] + out.stderr[-3000:]
+    lines = [l for l in out.stdout.splitlines() if l.strip().startswith("{")]
+    assert len(lines) == 1
+    r = json.loads(lines[0])
+    assert r["n_gpus"] == 1 and r["value"] > 0 and r["e2e"]["value"] > 0
+    assert r["config"]["T_per_gpu"] == 512 and r["config"]["slots_per_gpu"] == 8
+    assert r["independent_replicas"]["value"] > 0 and r["gpu_launches"] >= 40
