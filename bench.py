@@ -815,20 +815,28 @@ def run_group(args):
         replay, timed_how = g.replay, "CUDA-graph replays of one step"
     except Exception:
         torch.cuda.synchronize()
+    def timed_block():
+        dist.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(K):
+            replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return max_over_ranks(e0.elapsed_time(e1), world, dev)     # the same figure on every rank
+
     sampler = ClockSampler(local_rank)
-    dist.barrier()
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler.start()
-    e0.record()
-    for _ in range(K):
-        replay()
-    e1.record()
-    torch.cuda.synchronize()
+    block_ms = [timed_block()]
+    # every rank derives the same number of repeats from the same (max over ranks) first block
+    repeats = max(3, min(100, int(np.ceil(MIN_TIMED_SECONDS * 1e3 / block_ms[0]))))
+    while len(block_ms) < repeats:
+        block_ms.append(timed_block())
     clocks = sampler.stop()
     dist.barrier()
-    ms_total = max_over_ranks(e0.elapsed_time(e1), world, dev)
-    launches += 4 * K
+    ms_total = statistics.median(block_ms)
+    launches += 4 * K * len(block_ms)
     value = T * K / (ms_total * 1e-3)
 
     # end to end: every step uploads this rank's shard from pinned host memory and downloads its y
@@ -895,14 +903,16 @@ def run_group(args):
         alg = algorithmic_bytes(wl, T)
         print(json.dumps({
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
-            "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "strong" if world > 1 else "weak",
+            "ms_per_step": ms_total / K, "ms_per_step_min": min(block_ms) / K, "ms_per_step_max": max(block_ms) / K,
+            "timed_repeats": len(block_ms), "higher_is_better": True, "scaling": "strong" if world > 1 else "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {**base_config(wl, failed), "T_per_gpu": Tl, "slots_per_gpu": wl.P // world,
                        "parallelism": f"ep{world}: tokens sharded T/{world} per GPU, slots P/{world} per GPU; per step "
                                       "route, all-gather of per-slot counts (NCCL), scatter into the owners' receive "
                                       "buffers over peer memory, combine from them; two one-word all-reduces order the GPUs",
                        "l2": f"a step moves {sum(alg.values()) / 1e9:.2f} GB over all GPUs; inputs are not rotated",
-                       "timed": f"{timed_how}, CUDA events, max over ranks"},
+                       "timed": f"blocks of {K} steps, {timed_how}, CUDA events around each block, max over ranks per "
+                                f"block, blocks repeated until they span {MIN_TIMED_SECONDS} s, the median block is reported"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
             "roofline": {"bound": "hbm", "kernel": "step", "achieved": sum(alg.values()) * K / (ms_total * 1e-3) / 1e9,
                          "peak": measured_peaks()[0] * world, "unit": "GB/s",
