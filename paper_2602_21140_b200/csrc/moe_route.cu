@@ -42,6 +42,7 @@ struct Derived {
     int state_words;       // words of the whole routing-state blob
     int tokens_per_block;  // routing tile
     int p_pad;             // P rounded up to a multiple of 8 (row pitch of the per-tile counts)
+    bool alias_wcount;     // routing kernel: count matrix shares the token tables' shared memory
 };
 
 bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
@@ -114,10 +115,13 @@ bool derive(const moe_config *c, Derived *d, int want_lpt = 0, int want_tile = 0
     // a batch that one CTA routes in a single pass of its 32 warps needs no prefix over tiles at all
     if (want_tile <= 0 && c->max_tokens <= kRouteWarps * per_warp) tile = c->max_tokens;
     tile = (tile + per_warp - 1) / per_warp * per_warp;
+    // side by side if that fits with the smallest tile, else the count matrix shares the token tables
+    d->alias_wcount = route_smem_bytes(d->E, d->max_rep, per_warp, d->k, d->P, d->epl, false) > kMaxSmem - 1024;
+    const bool al = d->alias_wcount;
     while (tile > per_warp &&
-           (route_smem_bytes(d->E, d->max_rep, tile, d->k, d->P, d->epl) > kMaxSmem - 1024 || (long long)tile * d->k > 65535))
+           (route_smem_bytes(d->E, d->max_rep, tile, d->k, d->P, d->epl, al) > kMaxSmem - 1024 || (long long)tile * d->k > 65535))
         tile = (tile / 2 + per_warp - 1) / per_warp * per_warp;
-    if (route_smem_bytes(d->E, d->max_rep, tile, d->k, d->P, d->epl) > kMaxSmem - 1024 || (long long)tile * d->k > 65535)
+    if (route_smem_bytes(d->E, d->max_rep, tile, d->k, d->P, d->epl, al) > kMaxSmem - 1024 || (long long)tile * d->k > 65535)
         return false;
     d->tokens_per_block = tile;
     if ((c->max_tokens + tile - 1) / tile > kMaxRouteTiles) return false;
@@ -362,6 +366,7 @@ cudaError_t enqueue_route(moe_ctx *ctx, const float *logits, int32_t T, const mo
     rp.rank_counts = out->rank_counts; rp.rank_offsets = out->rank_offsets;
     rp.tile_counts = ctx->d_tile_counts; rp.ctl = ctx->d_ctl;
     rp.prefetch = ctx->pdl ? ctx->route_prefetch : 0;
+    rp.alias_wcount = d.alias_wcount ? 1 : 0;
     const int tiles = (T + d.tokens_per_block - 1) / d.tokens_per_block;
     return launch_route(d.epl, d.lpt, rp, tiles, ctx->route_smem, st, ctx->pdl);
 }
@@ -481,7 +486,7 @@ int tuned(const moe_ctx *ctx, int option, int dflt)
 void configure_launch(moe_ctx *ctx)
 {
     const Derived &d = ctx->d;
-    ctx->route_smem = route_smem_bytes(d.E, d.max_rep, d.tokens_per_block, d.k, d.P, d.epl);
+    ctx->route_smem = route_smem_bytes(d.E, d.max_rep, d.tokens_per_block, d.k, d.P, d.epl, d.alias_wcount);
     ctx->spin_limit = (unsigned)tuned(ctx, MOE_TUNE_SPIN_LIMIT, (int)kDefaultSpinLimit);
     ctx->pdl = tuned(ctx, MOE_TUNE_PDL, 1) != 0;
     ctx->scatter_impl = tuned(ctx, MOE_TUNE_SCATTER_IMPL, 0);

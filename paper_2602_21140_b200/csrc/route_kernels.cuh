@@ -89,22 +89,34 @@ struct RouteParams {
     int32_t *topk_slot;       // [T,k]
     int32_t *pos_in_slot;     // [T*k]: stable rank of assignment i inside its slot
     int32_t *slot_counts, *slot_offsets, *rank_counts, *rank_offsets;
+    int alias_wcount;         // the histogram's count matrix shares the token phase's tables (see route_smem_bytes)
     int prefetch;             // bit 0: ask the small tables into L2 before the wait; bit 1: the logits too
     ulonglong2 *tile_counts;  // [tiles][p_pad/4]: per tile, four slots to a 16-byte entry: two words
                               // of (epoch << 32 | count of the odd slot << 16 | count of the even slot)
     Control *ctl;
 };
 
+// Shared memory of the routing kernel.  The first region holds the per-warp tables of the token
+// phase ([blocks][32] 16-byte entries: logits, then key codes; [blocks][32] block bests).  The
+// per-warp count matrix of the histogram phase ([32][P] 16-bit) normally has a region of its own
+// and is zeroed before the kernel's wait; with very many slots or experts the two do not fit
+// side by side, and the matrix then shares the first region (`alias`), at the price of a
+// zeroing pass and a barrier between the two phases.
+__host__ __device__ inline size_t route_region0_words(int P, int epl, bool alias)
+{
+    const size_t code_words = (size_t)kRouteWarps * ((epl + 3) / 4) * 32 * 5;
+    const size_t count_words = alias ? ((size_t)kRouteWarps * P * sizeof(uint16_t) + 3) / 4 : 0;
+    return ((code_words > count_words ? code_words : count_words) + 3) & ~(size_t)3;
+}
+
 __host__ __device__ inline size_t route_smem_bytes(int E, int max_rep, int tokens_per_block, int k,
-                                                   int P, int epl)
+                                                   int P, int epl, bool alias)
 {
     const size_t p_pad = ((size_t)P + 7) & ~(size_t)7;
-    // per warp: [blocks][32] 16-byte entries (logits, then key codes) and [blocks][32] block bests
-    const size_t code_words = (size_t)kRouteWarps * ((epl + 3) / 4) * 32 * 5;
     const size_t bias_words = (size_t)((epl + 3) / 4 * 4) * 16 + 16;   // bias by (expert of the lane, lane); availability bits
-    size_t words = code_words + bias_words + (size_t)E * (1 + max_rep) + 2 * (size_t)tokens_per_block * k +
-                   2 * p_pad + (size_t)P;
-    return words * sizeof(int32_t) + (size_t)kRouteWarps * P * sizeof(uint16_t);
+    size_t words = route_region0_words(P, epl, alias) + bias_words + (size_t)E * (1 + max_rep) +
+                   2 * (size_t)tokens_per_block * k + 2 * p_pad + (size_t)P;
+    return words * sizeof(int32_t) + (alias ? 0 : (size_t)kRouteWarps * P * sizeof(uint16_t));
 }
 
 // Route 32/LPT tokens with one warp.  Lanes [sub*LPT, (sub+1)*LPT) own token
@@ -281,15 +293,17 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
     // bias of expert sl * EPL + q at s_bias[q * LPT + sl] (lanes of a token read neighbouring words),
     // zero past E; then 16 words of availability bits, bit e = expert e has a live replica
     constexpr int kBiasWords = (EPL + 3) / 4 * 4 * 16;
-    float *s_bias = reinterpret_cast<float *>(smem) + kRouteWarps * kBlockEntries * 5;
+    const int region0 = (int)route_region0_words(P, EPL, p.alias_wcount != 0);
+    float *s_bias = reinterpret_cast<float *>(smem) + region0;
     uint32_t *s_avail = reinterpret_cast<uint32_t *>(s_bias + kBiasWords);               // [16]
-    int32_t *s_live = smem + kRouteWarps * kBlockEntries * 5 + kBiasWords + 16;   // [E][1 + max_rep] live count, live slots
+    int32_t *s_live = smem + region0 + kBiasWords + 16;   // [E][1 + max_rep] live count, live slots
     int32_t *s_slot = s_live + E * live_words;        // [NA] slot of each assignment of the tile
     int32_t *s_lrank = s_slot + NA;                   // [NA] stable rank inside the tile
     int32_t *s_hist = s_lrank + NA;                   // [p_pad] tile histogram (running)
     int32_t *s_excl = s_hist + p.p_pad;               // [p_pad] assignments on slot p in earlier tiles
     int32_t *s_order = s_excl + p.p_pad;              // [P]  physical slot at each layout position
-    uint16_t *s_wcount = reinterpret_cast<uint16_t *>(s_order + P);  // [32][P] one round's counts
+    uint16_t *s_wcount = p.alias_wcount ? reinterpret_cast<uint16_t *>(smem)
+                                        : reinterpret_cast<uint16_t *>(s_order + P);  // [32][P] one round's counts
     __shared__ unsigned s_ticket, s_epoch;
     __shared__ int s_warp_sums[kRouteWarps];
 
@@ -301,8 +315,10 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
     // is paced by instruction fetch, and unrolled copies of once-run code only add to that.)
 #pragma unroll 1
     for (int q = tid; q < p.p_pad; q += kRouteThreads) { s_hist[q] = 0; s_excl[q] = 0; }
+    if (!p.alias_wcount) {
 #pragma unroll 1
-    for (int q = tid; q < kRouteWarps * P; q += kRouteThreads) s_wcount[q] = 0;
+        for (int q = tid; q < kRouteWarps * P; q += kRouteThreads) s_wcount[q] = 0;
+    }
 
     // ... apart from hints: under programmatic dependent launch this CTA may be resident well
     // before the previous kernel has finished, and the tables it is about to read were last
@@ -428,6 +444,12 @@ __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
         if (sl < k && lt < tb) s_slot[lt * k + sl] = slot;
     }
     __syncthreads();
+
+    if (p.alias_wcount) {                              // the token phase's tables are dead: reuse them
+#pragma unroll 1
+        for (int q = tid; q < kRouteWarps * P; q += kRouteThreads) s_wcount[q] = 0;
+        __syncthreads();
+    }
 
     // ---- tile histogram and stable rank of every assignment inside the tile 
     // Rounds of 1024 assignments in ascending i.  Inside a round, match_any gives

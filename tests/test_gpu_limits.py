@@ -64,6 +64,20 @@ def test_many_slots():
     run_and_check(wl, inp, (5, 77))
 
 
+@pytest.mark.parametrize("E,k,R,S", [(512, 8, 368, 8), (512, 8, 256, 4), (8, 2, 2900, 1)])
+def test_shapes_whose_routing_tables_share_shared_memory(E, k, R, S):
+    # so many slots or experts that the histogram's count matrix reuses the token phase's tables
+    P = R * S
+    assert B.moe_workspace_bytes(B.make_config(E, k, 64, 300, R, S, 1)) > 0
+    wl = W.Workload("edge", T=300, H=64, E=E, k=k, R=R, S=S, seed=51, max_replicas=1)
+    inp = W.make_inputs(dataclasses.replace(wl, R=max(E // 8, 1), S=8))     # logits / x / bias only
+    s2e = np.full(P, -1, np.int32)
+    s2e[np.linspace(0, P - 1, E).astype(int)] = np.arange(E)
+    inp["slot_to_expert"] = s2e
+    inp["slot_scale"] = np.random.default_rng(3).uniform(0.5, 1.5, P).astype(np.float32)
+    run_and_check(wl, inp, (1, 5))
+
+
 @pytest.mark.parametrize("max_tokens", [5000, 40000, 131072])
 def test_large_routing_tiles_and_partial_batches(max_tokens):
     # the routing tile grows with max_tokens (64 ... 1024 tokens); batches far below it still work
