@@ -782,88 +782,102 @@ def run_group(args):
     bias = inp["bias"] if wl.score_func == W.SIGMOID else None
     cfg = B.config_for_workload(wl, max_tokens=max(Tl, 1))
     recv_rows = T * wl.k                                # always suffices: every row of the step could land here
-    group = ep.DistributedEp(cfg, inp["slot_to_expert"], bias, inp["slot_scale"], recv_rows, dev)
-    apply_tuning(group.router, args.tune)
-    group.router.set_failed_ranks(failed)
-
-    lg_h = torch.from_numpy(inp["logits"][lo:hi]).pin_memory()
-    x_h = torch.from_numpy(inp["x"][lo:hi]).view(torch.int16).view(torch.bfloat16).pin_memory()
-    y_h = torch.empty((Tl, wl.H), dtype=torch.bfloat16).pin_memory()
-    logits, x = lg_h.to(dev), x_h.to(dev)
-    out = group.router.alloc_outputs(Tl)
-    out.send_buf = out.send_buf[:1]                    # no send buffer in this mode
-    y = torch.empty((Tl, wl.H), dtype=torch.bfloat16, device=dev)
-
-    def step():
-        group.dispatch(logits, x, out)
-        group.combine(Tl, y)
-
-    launches = 2
-    for _ in range(max(Wm, 3)):
-        step()
-    torch.cuda.synchronize()
-    launches += 4 * max(Wm, 3)
-    assert group.router.device_status() == 0
-    # a captured step (NCCL calls included) removes the host from the loop; plain launches otherwise
-    replay, timed_how = step, "eager launches"
+    # The exchange needs symmetric memory between the GPUs of the group.  Where that cannot be set
+    # up, every rank learns of it here (one all-reduce) and the run reports the independent
+    # replicas alone instead of failing half-way through a collective.
+    exch_error, group = None, None
     try:
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g):
+        group = ep.DistributedEp(cfg, inp["slot_to_expert"], bias, inp["slot_scale"], recv_rows, dev)
+    except Exception as exc:                            # noqa: BLE001 - reported in the JSON line
+        exch_error = f"{type(exc).__name__}: {exc}"[:300]
+    if max_over_ranks(1.0 if exch_error else 0.0, world, dev) > 0:
+        if group is not None:
+            group.close()
+        group = None
+        exch_error = exch_error or "another rank could not set up the exchange"
+    launches = 0
+    if group is not None:
+        apply_tuning(group.router, args.tune)
+        group.router.set_failed_ranks(failed)
+
+        lg_h = torch.from_numpy(inp["logits"][lo:hi]).pin_memory()
+        x_h = torch.from_numpy(inp["x"][lo:hi]).view(torch.int16).view(torch.bfloat16).pin_memory()
+        y_h = torch.empty((Tl, wl.H), dtype=torch.bfloat16).pin_memory()
+        logits, x = lg_h.to(dev), x_h.to(dev)
+        out = group.router.alloc_outputs(Tl)
+        out.send_buf = out.send_buf[:1]                    # no send buffer in this mode
+        y = torch.empty((Tl, wl.H), dtype=torch.bfloat16, device=dev)
+
+        def step():
+            group.dispatch(logits, x, out)
+            group.combine(Tl, y)
+
+        launches = 2
+        for _ in range(max(Wm, 3)):
             step()
-        g.replay()
         torch.cuda.synchronize()
-        replay, timed_how = g.replay, "CUDA-graph replays of one step"
-    except Exception:
-        torch.cuda.synchronize()
-    def timed_block():
+        launches += 4 * max(Wm, 3)
+        assert group.router.device_status() == 0
+        # a captured step (NCCL calls included) removes the host from the loop; plain launches otherwise
+        replay, timed_how = step, "eager launches"
+        try:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                step()
+            g.replay()
+            torch.cuda.synchronize()
+            replay, timed_how = g.replay, "CUDA-graph replays of one step"
+        except Exception:
+            torch.cuda.synchronize()
+        def timed_block():
+            dist.barrier()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(K):
+                replay()
+            e1.record()
+            torch.cuda.synchronize()
+            return max_over_ranks(e0.elapsed_time(e1), world, dev)     # the same figure on every rank
+
+        sampler = ClockSampler(local_rank)
+        sampler.start()
+        block_ms = [timed_block()]
+        # every rank derives the same number of repeats from the same (max over ranks) first block
+        repeats = max(3, min(100, int(np.ceil(MIN_TIMED_SECONDS * 1e3 / block_ms[0]))))
+        while len(block_ms) < repeats:
+            block_ms.append(timed_block())
+        clocks = sampler.stop()
         dist.barrier()
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(K):
-            replay()
-        e1.record()
-        torch.cuda.synchronize()
-        return max_over_ranks(e0.elapsed_time(e1), world, dev)     # the same figure on every rank
+        ms_total = statistics.median(block_ms)
+        launches += 4 * K * len(block_ms)
+        value = T * K / (ms_total * 1e-3)
 
-    sampler = ClockSampler(local_rank)
-    sampler.start()
-    block_ms = [timed_block()]
-    # every rank derives the same number of repeats from the same (max over ranks) first block
-    repeats = max(3, min(100, int(np.ceil(MIN_TIMED_SECONDS * 1e3 / block_ms[0]))))
-    while len(block_ms) < repeats:
-        block_ms.append(timed_block())
-    clocks = sampler.stop()
-    dist.barrier()
-    ms_total = statistics.median(block_ms)
-    launches += 4 * K * len(block_ms)
-    value = T * K / (ms_total * 1e-3)
+        # end to end: every step uploads this rank's shard from pinned host memory and downloads its y
+        K3 = min(K, 20)
+        lg_d, x_d = torch.empty_like(logits), torch.empty_like(x)
 
-    # end to end: every step uploads this rank's shard from pinned host memory and downloads its y
-    K3 = min(K, 20)
-    lg_d, x_d = torch.empty_like(logits), torch.empty_like(x)
+        def host_step():
+            lg_d.copy_(lg_h, non_blocking=True)
+            x_d.copy_(x_h, non_blocking=True)
+            group.dispatch(lg_d, x_d, out)
+            group.combine(Tl, y)
+            y_h.copy_(y, non_blocking=True)
+            torch.cuda.synchronize()
 
-    def host_step():
-        lg_d.copy_(lg_h, non_blocking=True)
-        x_d.copy_(x_h, non_blocking=True)
-        group.dispatch(lg_d, x_d, out)
-        group.combine(Tl, y)
-        y_h.copy_(y, non_blocking=True)
-        torch.cuda.synchronize()
-
-    for _ in range(2):
-        host_step()
-    dist.barrier()
-    t0 = time.perf_counter()
-    for _ in range(K3):
-        host_step()
-    e2e_s = max_over_ranks(time.perf_counter() - t0, world, dev)
-    launches += 4 * (K3 + 2)
-    e2e = {"value": T * K3 / e2e_s, "unit": UNIT, "h2d_bytes_per_step": T * wl.E * 4 + T * wl.H * 2,
-           "d2h_bytes_per_step": T * wl.H * 2, "steps": K3, "ms_per_step": 1e3 * e2e_s / K3,
-           "what": "bytes are whole-job totals over all ranks; each rank moves its T/N shard"}
-    assert group.router.device_status() == 0
-    group.close()
+        for _ in range(2):
+            host_step()
+        dist.barrier()
+        t0 = time.perf_counter()
+        for _ in range(K3):
+            host_step()
+        e2e_s = max_over_ranks(time.perf_counter() - t0, world, dev)
+        launches += 4 * (K3 + 2)
+        e2e = {"value": T * K3 / e2e_s, "unit": UNIT, "h2d_bytes_per_step": T * wl.E * 4 + T * wl.H * 2,
+               "d2h_bytes_per_step": T * wl.H * 2, "steps": K3, "ms_per_step": 1e3 * e2e_s / K3,
+               "what": "bytes are whole-job totals over all ranks; each rank moves its T/N shard"}
+        assert group.router.device_status() == 0
+        group.close()
 
     # extra: N independent replicas, every rank a whole batch of its own and no exchange (weak scaling)
     inp_r = W.make_inputs(wl, T=T, seed=shard_seed(wl.seed, rank))
@@ -899,7 +913,18 @@ def run_group(args):
     assert router.device_status() == 0
     router.close()
 
-    if rank == 0:
+    if rank == 0 and group is None:
+        # no exchange on this machine: the replicas are all there is to report
+        print(json.dumps({
+            "metric": METRIC, "value": replicas["value"], "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+            "ms_per_step": replicas["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {**base_config(wl, failed), "T_per_gpu": T,
+                       "parallelism": f"{world} independent replicas, no data-path collective",
+                       "timed": "CUDA-graph replays of one step, CUDA events, max over ranks"},
+            "exchange_unavailable": exch_error, "clocks": None, "e2e": None, "gpu_launches": launches,
+            "roofline": None, "cpu_baseline": None, "independent_replicas": replicas}))
+    elif rank == 0:
         alg = algorithmic_bytes(wl, T)
         print(json.dumps({
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
