@@ -5,11 +5,13 @@
 // Work split: a CTA of 32 warps takes one tile of `tokens_per_block` consecutive
 // tokens (tiles are handed out by an atomic ticket, so every tile a CTA may wait
 // for is already running).  A warp routes 32/LPT tokens at once: a token owns
-// LPT consecutive lanes and lane s of them holds experts [s*EPL, (s+1)*EPL) in
-// registers, which makes "lower lane" equal "lower expert id" for tie-breaks,
-// puts a whole expert group inside a power-of-two run of lanes, and keeps every
-// lane busy in the serial top-k rounds (the kernel is bound by instruction
-// issue, not by memory).
+// LPT consecutive lanes and lane s of them holds experts [s*EPL, (s+1)*EPL) (in
+// its own column of a shared-memory table), which makes "lower lane" equal
+// "lower expert id" for tie-breaks, puts a whole expert group inside a
+// power-of-two run of lanes, and keeps every lane busy in the serial top-k
+// rounds.  The kernel is bound by latency — instruction fetch, shared-memory
+// conflicts, trips to L2 — not by arithmetic or DRAM, and is written accordingly:
+// rolled loops, conflict-free tables, few dependent round trips.
 //
 // Prefix over tiles: the whole problem fits in one wave of CTAs (the host sizes the
 // tile so that a step has about one tile per SM), so all tiles publish at about the
@@ -282,7 +284,7 @@ __device__ __forceinline__ void route_tokens(const RouteParams &p, int t_first, 
 template <int EPL, int LPT>
 __global__ void __launch_bounds__(kRouteThreads, 1) k_route(RouteParams p)
 {
-    extern __shared__ int32_t smem[];
+    extern __shared__ __align__(16) int32_t smem[];
     const int E = p.E, P = p.P, k = p.k, tb = p.tokens_per_block;
     const int NA = tb * k;
     const int live_words = 1 + p.max_rep;
