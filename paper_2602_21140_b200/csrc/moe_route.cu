@@ -86,7 +86,13 @@ bool derive(const moe_config *c, Derived *d, int want_lpt = 0, int want_tile = 0
     }
     // 16 lanes per token above 64 experts: twice the warps in flight for the same work,
     // which measured faster than 8 lanes (the kernel is issue/latency bound)
-    if (want_lpt != 8 && want_lpt != 16) want_lpt = (d->E > 64) ? 16 : 0;
+    // ... as long as a tile is then routed in one pass of the CTA's warps (64 tokens with 16
+    // lanes each).  Larger tiles take several passes, each of which waits for its logits anew;
+    // eight lanes per token route 128 tokens per pass and win there (-3 us per step at 16384
+    // tokens and 128 experts, -7 us at 32768), so they are tried first when the shape allows them.
+    const int tile_tokens = want_tile > 0 ? want_tile
+                                          : std::max(32, (c->max_tokens + kRouteTileTarget - 1) / kRouteTileTarget);
+    if (want_lpt != 8 && want_lpt != 16) want_lpt = (d->E > 64 && tile_tokens <= 64) ? 16 : 0;
     for (int lpt : kLpt) {
         if (d->epl || d->k > lpt || (want_lpt && lpt < want_lpt)) continue;
         for (int epl : kEpl) {
