@@ -122,3 +122,28 @@ def test_routing_tables_around_the_default_shared_memory_limit(R):
     inp["slot_to_expert"] = s2e
     inp["slot_scale"] = np.random.default_rng(4).uniform(0.5, 1.5, R * S).astype(np.float32)
     run_and_check(wl, inp, (1, 40))
+
+
+def test_tuning_call_validates_and_restores():
+    wl = W.WORKLOADS["dsv3"]
+    inp = W.make_inputs(wl, T=300, H=128)
+    router = B.MoeRouter(B.config_for_workload(wl, max_tokens=300, hidden=128), inp["slot_to_expert"],
+                         inp["bias"], inp["slot_scale"])
+    ctx = router._ctx
+    assert B.moe_set_tuning(ctx, -1, 0) == B.MOE_ERR_INVALID_ARG
+    assert B.moe_set_tuning(ctx, 99, 0) == B.MOE_ERR_INVALID_ARG
+    assert B.moe_set_tuning(ctx, B.MOE_TUNE_PDL, -2) == B.MOE_ERR_INVALID_ARG
+    assert B.moe_set_tuning(None, B.MOE_TUNE_PDL, 0) == B.MOE_ERR_INVALID_ARG
+    # a tile the shape cannot have (not enough shared memory for it) is refused and nothing changes
+    assert B.moe_set_tuning(ctx, B.MOE_TUNE_ROUTE_TOKENS_PER_TILE, 10 ** 6) in (B.MOE_OK, B.MOE_ERR_INVALID_ARG)
+    run_and_check(wl, inp, (), router=router)
+    # overrides, then back to the automatic choices: results never change
+    for option, value in ((B.MOE_TUNE_ROUTE_TOKENS_PER_TILE, 16), (B.MOE_TUNE_COMBINE_IMPL, 0),
+                          (B.MOE_TUNE_SCATTER_IMPL, 1), (B.MOE_TUNE_ROUTE_PREFETCH, 0),
+                          (B.MOE_TUNE_SCATTER_STORE_POLICY, 3)):
+        assert B.moe_set_tuning(ctx, option, value) == B.MOE_OK
+        run_and_check(wl, inp, (), router=router)
+    for option in range(16):
+        assert B.moe_set_tuning(ctx, option, -1) == B.MOE_OK
+    run_and_check(wl, inp, (), router=router)
+    router.close()
