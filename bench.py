@@ -517,7 +517,7 @@ def run_single(args):
         value = T * K / (ms_total * 1e-3)
 
         # ---- per-kernel durations: eager launches with events between the kernels
-        K2 = min(max(K, 50), 200)
+        K2 = 200
         ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K2)]
         for i in range(K2):
             router.set_timing_event(ev[i][1])
